@@ -1,0 +1,333 @@
+#!/usr/bin/env python
+"""Benchmark of the zero-expert MoE layer forward (one step = one zeda_moe_forward call over one
+batch of synthetic tokens: router, top-K, compaction, grouped SwiGLU experts, combine).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload decode|prefill|sweep25|...]
+    python bench.py --impl reference ...      # the CPU oracle, timed on the host cores
+
+Prints ONE JSON line.  With N > 1 (launched by torch.distributed.run) every rank is a data-parallel
+replica of the layer with its own token batch; there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2605_18643_b200 import flops, inputs
+
+METRIC = "MoE-layer tokens/s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def make_workload(name: str):
+    if name == "decode":
+        return inputs.decode()
+    if name == "prefill":
+        return inputs.prefill()
+    if name == "tiny":
+        return inputs.tiny()
+    if name.startswith("sweep"):
+        return inputs.sweep_point(int(name[5:]) / 100.0)
+    if name.startswith("prefill_f"):   # zero-fraction sweep at the prefill size
+        f = int(name[9:]) / 100.0
+        return inputs.prefill(Z=0, zero_fraction=None) if f == 0 else inputs.prefill(zero_fraction=f)
+    raise SystemExit("unknown workload " + name)
+
+
+def workload_config(wl, name, extra=None):
+    c = {"workload": name, "T": wl.T, "d": wl.d, "d_expert": wl.He, "n_real": wl.E, "n_zero": wl.Z,
+         "top_k": wl.K, "zero_slot_fraction": round(wl.zero_fraction, 4), "seed": 0}
+    if extra:
+        c.update(extra)
+    return c
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "--id=%d" % self.index, "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [v.strip() for v in line.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, f[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def oracle_tokens_per_s(wl, sample_tokens: int, seed: int = 0):
+    """Times the CPU oracle, as it stands, on a bounded token sample of the workload."""
+    import oracle
+    n = min(sample_tokens, wl.T)
+    ids = None if n == wl.T else np.sort(np.random.default_rng(seed).choice(wl.T, n, replace=False)).astype(np.int32)
+    bias = None if wl.router_bias is None else wl.router_bias.numpy()
+    args = (inputs.bits(wl.x), wl.router_w.numpy(), bias, inputs.bits(wl.w_gate_up), inputs.bits(wl.w_down),
+            wl.E, wl.Z, wl.K)
+    t0 = time.perf_counter()
+    oracle.forward(*args, token_ids=ids)
+    dt = time.perf_counter() - t0
+    sample = "%d of %d tokens, seeded sample, 1 pass" % (n, wl.T) if ids is not None else "all %d tokens, 1 pass" % wl.T
+    return n / dt, dt, oracle.num_threads(), sample
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores, same metric and workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = make_workload(args.workload)
+    sample = 64 if wl.T > 64 else wl.T
+    for _ in range(min(args.warmup, 1)):
+        oracle_tokens_per_s(wl, sample)
+    times, tps = [], []
+    steps = max(1, min(args.steps, 5))
+    info = None
+    for _ in range(steps):
+        v, dt, cores, desc = oracle_tokens_per_s(wl, sample)
+        times.append(dt)
+        tps.append(v)
+        info = (cores, desc)
+    total = sum(times)
+    value = sample * steps / total
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * total / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(wl, args.workload, {"note": "each step = the oracle on a bounded token sample"}),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": info[0], "kind": "oracle", "sample": info[1]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def time_forward(m, x, y, steps, warmup, flush, dist_barrier):
+    """Per-step CUDA-event timing with an L2 flush (outside the event pairs) between steps."""
+    for _ in range(warmup):
+        flush.zero_()
+        m.forward(x, y)
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    dist_barrier()
+    torch.cuda.synchronize()
+    for i in range(steps):
+        flush.zero_()
+        starts[i].record()
+        m.forward(x, y)
+        ends[i].record()
+    torch.cuda.synchronize()
+    dist_barrier()
+    per = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    return sum(per), per
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="decode")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-static", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group(backend="nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    from paper_2605_18643_b200 import zeda  # raises if libzeda.so is missing
+
+    peaks, peaks_kind = load_peaks()
+    wl = make_workload(args.workload)
+    x_cpu = wl.x if rank == 0 else inputs.replica_tokens(wl, rank)
+    m = zeda.from_workload(wl, dev)
+    x = x_cpu.to(dev)
+    y = torch.empty_like(x)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    clocks = ClockSampler(local_rank)
+    clocks.start()
+    total_ms, per = time_forward(m, x, y, args.steps, args.warmup, flush, barrier)
+    P, U, zero_slots, launches = m.last_counters()
+
+    # the same steps again with stage events on the stream: duration of the dominant kernel
+    m.set_profiling(True)
+    stage = np.zeros(5)
+    for i in range(args.steps):
+        flush.zero_()
+        m.forward(x, y)
+        stage += np.array(m.stage_ms())
+    stage /= args.steps
+    m.set_profiling(False)
+
+    # end to end through the host-buffer entry point: H2D of x and D2H of y inside the timed region
+    x_pin = x_cpu.pin_memory()
+    y_pin = torch.empty_like(x_pin).pin_memory()
+    for _ in range(args.warmup):
+        flush.zero_()
+        m.forward_host(x_pin, y_pin)
+    barrier()
+    torch.cuda.synchronize()
+    e2e_s = 0.0
+    for i in range(args.steps):
+        flush.zero_()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        m.forward_host(x_pin, y_pin)
+        e2e_s += time.perf_counter() - t0
+    barrier()
+    clock_info = clocks.stop()
+
+    # static top-K reference: the same kernels with the zero experts removed (Z = 0)
+    static = None
+    if not args.no_static and wl.Z > 0:
+        ws = inputs.static_reference(wl)
+        ms_ = zeda.from_workload(ws, dev)
+        st_total, _ = time_forward(ms_, x, y, args.steps, args.warmup, flush, barrier)
+        Ps, Us, _, _ = ms_.last_counters()
+        ms_.close()
+        static = {"ms_per_step": st_total / args.steps, "P": Ps, "U": Us}
+
+    # max over ranks
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_s, static["ms_per_step"] if static else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_s = float(t[0]), float(t[1])
+        if static:
+            static["ms_per_step"] = float(t[2])
+
+    if rank == 0:
+        ms_per_step = total_ms / args.steps
+        value = world * wl.T / (ms_per_step * 1e-3)
+        hbm = peaks["hbm_gbs"] * 1e9
+        n_cand = wl.E + wl.Z
+        t_roof, t_flop, t_mem = flops.layer_roofline_seconds(wl.T, wl.d, wl.He, n_cand, P, U,
+                                                             peaks["bf16_tflops"] * 1e12, hbm)
+        # dominant kernel: expert GEMM1 + SwiGLU; algorithmic bytes = gate and up weights of the U
+        # active experts + the x rows it reads + the intermediate it writes
+        names = ["router", "sort", "gemm1", "gemm2", "combine"]
+        g1_bytes = U * 2 * wl.He * wl.d * 2 + wl.T * wl.d * 2 + P * wl.He * 2
+        g1_flops = 4 * P * wl.d * wl.He
+        g1_s = stage[2] * 1e-3
+        hbm_bound = g1_bytes / hbm >= g1_flops / (peaks["bf16_tflops"] * 1e12)
+        if hbm_bound:
+            roof = {"bound": "hbm", "achieved": g1_bytes / g1_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        else:
+            roof = {"bound": "tensor", "achieved": g1_flops / g1_s / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof.update(traffic=None, kernel="expert GEMM1 + SwiGLU", peak_source=peaks_kind,
+                    algorithmic_bytes=g1_bytes, algorithmic_flops=g1_flops, kernel_ms=stage[2])
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_config(wl, args.workload, {
+                "P": P, "U": U, "l2": "256 MiB buffer written between timed steps (outside the event pairs)",
+                "parallelism": "dp%d replicas, no collective" % world}),
+            "clocks": clock_info,
+            "e2e": {"value": world * wl.T * args.steps / e2e_s, "unit": UNIT,
+                    "h2d_bytes_per_step": wl.T * wl.d * 2, "d2h_bytes_per_step": wl.T * wl.d * 2,
+                    "ms_per_step": 1e3 * e2e_s / args.steps},
+            "gpu_launches": launches * args.steps,
+            "roofline": roof,
+            "layer_roofline": {"t_roof_us": t_roof * 1e6, "t_flop_us": t_flop * 1e6, "t_hbm_us": t_mem * 1e6,
+                               "frac": t_roof / (ms_per_step * 1e-3), "peak_source": peaks_kind},
+            "stage_ms": {n: float(v) for n, v in zip(names, stage)},
+        }
+        if static:
+            line["static_reference"] = dict(static, value=world * wl.T / (static["ms_per_step"] * 1e-3),
+                                            speedup_vs_static=static["ms_per_step"] / ms_per_step)
+        if not args.no_cpu_baseline:
+            v, dt, cores, desc = oracle_tokens_per_s(wl, 64)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+                                    "seconds": dt}
+        print(json.dumps(line))
+    m.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

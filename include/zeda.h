@@ -1,0 +1,175 @@
+/*
+ * zeda.h - C ABI of the B200 (sm_100a) forward pass of an MoE layer with zero-output experts.
+ *
+ * The layer (paper Section 2.1 "Zero-Expert Injection", Eq. 1): a router scores N normal experts
+ * and N_Z zero experts (Z_j(h) = 0), keeps the top-K of the union, and the output is
+ *     y~(h) = sum over the selected slots that are normal experts of g~_i(h) * E_i(h),
+ * with the routing weights of the surviving slots left as they were (Section 4.3.4: no
+ * renormalisation; Eq. 7 is the renormalised variant).  Each expert has gate, up and down
+ * projections (Appendix D), read here as down(silu(gate x) * up x).
+ *
+ * Conventions
+ *   - Candidate ids: 0..N-1 normal experts, N..N+N_Z-1 zero experts (E' = E u Z).
+ *   - "dev" pointers are CUDA device pointers on the handle's device, "host" pointers are host
+ *     memory.  The caller owns every buffer it passes (weights, workspace, inputs, outputs) and
+ *     keeps weights and workspace alive and unmodified until zeda_moe_destroy.  The library never
+ *     allocates, frees or resizes device memory.
+ *   - bf16 tensors are passed as const void* / void* (16-bit patterns), row-major, 16-byte aligned.
+ *   - Calls enqueue work on the given cudaStream_t (passed as void*, NULL = default stream) and
+ *     return without synchronising, except where stated.  Outputs are valid once the stream has
+ *     been synchronised.  A handle is not thread-safe; distinct handles are independent.
+ *   - Every entry point returns a zeda_status_t (ZEDA_OK = 0); nothing throws, aborts or traps.
+ *     Arguments are checked before anything is launched; zeda_last_error() gives a text for the
+ *     last failure on the calling thread.
+ */
+#ifndef ZEDA_H_
+#define ZEDA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct zeda_moe zeda_moe_t; /* opaque; host memory owned by the library */
+
+typedef enum {
+    ZEDA_OK = 0,
+    ZEDA_ERR_INVALID_ARG = -1, /* null/misaligned pointer, bad size, T > max_tokens, ... */
+    ZEDA_ERR_UNSUPPORTED = -2, /* a shape the kernels do not cover (see zeda_moe_config_t) */
+    ZEDA_ERR_WORKSPACE = -3,   /* workspace smaller than zeda_moe_workspace_bytes() */
+    ZEDA_ERR_CUDA = -4,        /* a CUDA runtime call failed; text in zeda_last_error() */
+    ZEDA_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (reported by a later call) */
+} zeda_status_t;
+
+/* How the routing weight g~ of a selected slot is formed from p = softmax(logits over N+N_Z).
+ * The paper says "normalized routing weight" (Section 2.1) without giving the formula. */
+typedef enum {
+    ZEDA_GATE_TOPK_NORM = 0,   /* p_i / sum of p over the K selected slots (zero slots included
+                                  in the sum); default */
+    ZEDA_GATE_SOFTMAX_RAW = 1, /* p_i itself */
+    ZEDA_GATE_RENORM_REAL = 2  /* Eq. 7: p_i / sum of p over the selected NORMAL experts; zero
+                                  slots get weight 0 */
+} zeda_gate_mode_t;
+
+/* What an injected expert outputs. */
+typedef enum {
+    ZEDA_EXPERT_ZERO = 0, /* Z_j(h) = 0 (Section 2.1) */
+    ZEDA_EXPERT_COPY = 1  /* copy expert of Appendix B: adds (sum of zero-slot weights) * h */
+} zeda_expert_kind_t;
+
+/* Supported shapes: d_model and d_expert multiples of 64 in [64, 8192], 1 <= top_k <= 16,
+ * n_real >= 1, n_zero >= 0, n_real + n_zero <= 512, top_k <= n_real + n_zero,
+ * max_tokens >= 1 and max_tokens * top_k < 2^27. */
+typedef struct {
+    int32_t d_model;     /* H: hidden size */
+    int32_t d_expert;    /* H_e: expert intermediate size */
+    int32_t n_real;      /* N: normal experts */
+    int32_t n_zero;      /* N_Z: zero experts (0 = the static top-K layer) */
+    int32_t top_k;       /* K */
+    int32_t max_tokens;  /* largest T any call will pass */
+    int32_t gate_mode;   /* zeda_gate_mode_t */
+    int32_t expert_kind; /* zeda_expert_kind_t */
+    int32_t device;      /* CUDA device ordinal */
+    int32_t flags;       /* ZEDA_FLAG_* */
+} zeda_moe_config_t;
+
+enum {
+    ZEDA_FLAG_NONE = 0,
+    ZEDA_FLAG_FORCE_STREAM_EXPERTS = 1, /* always use the weight-streaming expert kernels */
+    ZEDA_FLAG_FORCE_TILE_EXPERTS = 2    /* always use the tcgen05 tile kernels */
+};
+
+/* Device workspace the handle needs for the given configuration (bytes, multiple of 256);
+ * 0 if the configuration is invalid. */
+size_t zeda_moe_workspace_bytes(const zeda_moe_config_t *cfg);
+
+/* Builds a handle.  Section 2.1: the router has N + N_Z rows.
+ *   router_w     dev [N+N_Z, d_model] fp32, rows 0..N-1 normal, N.. zero experts
+ *   router_bias  dev [N+N_Z] fp32 added to the logits, or NULL (the paper's layer has none)
+ *   w_gate_up    dev [N, 2*d_expert, d_model] bf16; per expert rows 0..H_e-1 = gate, H_e.. = up
+ *   w_down       dev [N, d_model, d_expert] bf16
+ *   workspace    dev, >= zeda_moe_workspace_bytes(cfg), 256-byte aligned; the library carves it
+ * Makes the configured device current, may launch a one-time set-up kernel on the default stream
+ * and synchronises before returning. */
+zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_w,
+                              const float *router_bias, const void *w_gate_up, const void *w_down,
+                              void *workspace, size_t workspace_bytes, zeda_moe_t **out);
+
+/* Routing only (Section 2.1: top-K over E'; zero slots dropped; surviving pairs grouped by expert).
+ *   x               dev [T, d_model] bf16
+ *   topk_idx        dev [T, K] int32: candidates in descending logit order, ties to the lower id
+ *   topk_w          dev [T, K] fp32 routing weights per gate_mode
+ *   expert_counts   dev [N] int32 pairs per normal expert
+ *   expert_offsets  dev [N+1] int32 exclusive prefix sum; [N] = P
+ *   perm            dev [T*K] int32; the first P entries list the surviving slots t*K+k ordered by
+ *                   (expert ascending, token ascending); the rest is left untouched
+ *   n_pairs         dev [1] int32 = P
+ * Any output pointer may be NULL.  T == 0 returns ZEDA_OK and touches nothing. */
+zeda_status_t zeda_route(zeda_moe_t *h, const void *x, int32_t T, int32_t *topk_idx, float *topk_w,
+                         int32_t *expert_counts, int32_t *expert_offsets, int32_t *perm,
+                         int32_t *n_pairs, void *stream);
+
+/* Test entry: as zeda_route, but the top-K is taken over caller-supplied fp32 logits
+ * dev [T, N+N_Z] instead of x * router_w^T + bias. */
+zeda_status_t zeda_route_from_logits(zeda_moe_t *h, const float *logits, int32_t T,
+                                     int32_t *topk_idx, float *topk_w, int32_t *expert_counts,
+                                     int32_t *expert_offsets, int32_t *perm, int32_t *n_pairs,
+                                     void *stream);
+
+/* Test entry: the fp32 router logits x * router_w^T + bias, dev [T, N+N_Z]. */
+zeda_status_t zeda_router_logits(zeda_moe_t *h, const void *x, int32_t T, float *logits, void *stream);
+
+/* Layer forward, Eq. 1 (Eq. 7 / Appendix B through the configured modes).
+ *   x  dev [T, d_model] bf16      y  dev [T, d_model] bf16, fully overwritten
+ * A token whose K slots all fall on zero experts gets exact +0 in every element of its row.
+ * x and y must not overlap.  T == 0 returns ZEDA_OK and touches nothing. */
+zeda_status_t zeda_moe_forward(zeda_moe_t *h, const void *x, int32_t T, void *y, void *stream);
+
+/* The same forward for callers whose activations live in HOST memory: copies x to the device,
+ * runs the layer, copies y back, all on `stream`, and synchronises the stream before returning.
+ *   x_host  host [T, d_model] bf16     y_host  host [T, d_model] bf16
+ * Pinned host memory makes the copies asynchronous; pageable memory works but is slower. */
+zeda_status_t zeda_moe_forward_host(zeda_moe_t *h, const void *x_host, int32_t T, void *y_host,
+                                    void *stream);
+
+/* Routing statistics of the most recent zeda_route / zeda_moe_forward call on this handle
+ * (Section 2.2, Eq. 4-6), computed on the device from that call's routing:
+ *   f      dev [N+N_Z] fp32  share of tokens whose top-K set holds candidate i (f_i), or NULL
+ *   p_mean dev [N+N_Z] fp32  mean softmax probability of candidate i over the batch (P_i), or NULL
+ *   out    dev [4] fp32      {r_ZE, sum_i f_i P_i, f_E P_E, f_Z P_Z}; the caller scales these into
+ *                            L_A and L_GA with its alpha and w
+ * Needs the logits, so it re-runs the router on x. */
+zeda_status_t zeda_moe_stats(zeda_moe_t *h, const void *x, int32_t T, float *f, float *p_mean,
+                             float *out, void *stream);
+
+/* Counters of the last forward call, read back after synchronising the stream (blocking):
+ * out[0] = P (surviving pairs), out[1] = U (normal experts with at least one pair),
+ * out[2] = zero-expert slots, out[3] = kernels launched by that call. */
+zeda_status_t zeda_moe_last_counters(zeda_moe_t *h, int64_t out[4], void *stream);
+
+/* Per-stage device timing for measurement.  With profiling enabled, every later forward call
+ * records CUDA events on its stream between the stages; zeda_moe_stage_ms synchronises on the
+ * events of the last forward call (blocking) and returns the elapsed milliseconds of
+ * {router logits, top-K + counting sort, expert GEMM1 + SwiGLU, expert GEMM2, combine}.
+ * Enabling creates host-side event objects only (no device memory). */
+enum { ZEDA_STAGE_ROUTER = 0, ZEDA_STAGE_SORT = 1, ZEDA_STAGE_GEMM1 = 2, ZEDA_STAGE_GEMM2 = 3,
+       ZEDA_STAGE_COMBINE = 4, ZEDA_STAGE_COUNT = 5 };
+zeda_status_t zeda_moe_set_profiling(zeda_moe_t *h, int32_t enable);
+zeda_status_t zeda_moe_stage_ms(zeda_moe_t *h, float ms[ZEDA_STAGE_COUNT]);
+
+/* Reports a pending device-side error word (ZEDA_ERR_TIMEOUT) if any, then releases the handle.
+ * Does not touch caller-owned device memory. */
+zeda_status_t zeda_moe_destroy(zeda_moe_t *h);
+
+/* Text of the last failure on the calling thread ("" if none). Never NULL. */
+const char *zeda_last_error(void);
+
+/* Library version string. */
+const char *zeda_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZEDA_H_ */

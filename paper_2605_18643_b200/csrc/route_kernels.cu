@@ -1,0 +1,433 @@
+// Routing stage: router logits over the N + N_Z candidates, softmax / top-K / routing weights
+// (Section 2.1), then the compaction that drops zero-expert slots and counting-sorts the surviving
+// (token, normal expert) pairs by expert in a stable order.
+#include "zeda_internal.h"
+
+namespace zeda {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Router logits, CUDA-core version: l[t, j] = <x_t, W_r[j]> + b[j] in fp32.
+// One CTA = kTok tokens (bf16 rows staged in shared memory) x a slice of the candidates; one warp
+// per candidate row, lanes striding the feature axis with 16-byte loads.
+// ---------------------------------------------------------------------------------------------
+constexpr int kTok = 8;
+
+__global__ void __launch_bounds__(256)
+router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ router_w,
+                     const float *__restrict__ router_bias, int T, int d, int n_cand,
+                     int cand_per_cta, float *__restrict__ logits) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __nv_bfloat16 *xs = reinterpret_cast<__nv_bfloat16 *>(smem_raw);  // [kTok][d]
+    const int t0 = blockIdx.x * kTok;
+    const int nt = min(kTok, T - t0);
+    const int vec_per_row = d / 8;
+    for (int i = threadIdx.x; i < kTok * vec_per_row; i += blockDim.x) {
+        const int r = i / vec_per_row, c = i % vec_per_row;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (r < nt) v = __ldg(reinterpret_cast<const uint4 *>(x + (size_t)(t0 + r) * d) + c);
+        reinterpret_cast<uint4 *>(xs + (size_t)r * d)[c] = v;
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int j_begin = blockIdx.y * cand_per_cta;
+    const int j_end = min(n_cand, j_begin + cand_per_cta);
+    for (int j = j_begin + warp; j < j_end; j += 8) {
+        float acc[kTok];
+#pragma unroll
+        for (int r = 0; r < kTok; ++r) acc[r] = 0.f;
+        const float4 *wrow = reinterpret_cast<const float4 *>(router_w + (size_t)j * d);
+        for (int c4 = lane; c4 < d / 4; c4 += 32) {
+            const float4 w = __ldg(wrow + c4);
+#pragma unroll
+            for (int r = 0; r < kTok; ++r) {
+                const uint2 xv = reinterpret_cast<const uint2 *>(xs + (size_t)r * d)[c4];
+                const float x0 = __uint_as_float(xv.x << 16), x1 = __uint_as_float(xv.x & 0xffff0000u);
+                const float x2 = __uint_as_float(xv.y << 16), x3 = __uint_as_float(xv.y & 0xffff0000u);
+                acc[r] = fmaf(w.x, x0, acc[r]);
+                acc[r] = fmaf(w.y, x1, acc[r]);
+                acc[r] = fmaf(w.z, x2, acc[r]);
+                acc[r] = fmaf(w.w, x3, acc[r]);
+            }
+        }
+        const float b = router_bias ? __ldg(router_bias + j) : 0.f;
+#pragma unroll
+        for (int r = 0; r < kTok; ++r) {
+            const float s = warp_sum(acc[r]);
+            if (lane == 0 && r < nt) logits[(size_t)(t0 + r) * n_cand + j] = s + b;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Softmax, top-K and routing weights: one warp per token, logits held in registers (candidate
+// j lives in lane j % 32, register j / 32).  K rounds of warp arg-max; equal logits go to the
+// lower candidate id.
+// ---------------------------------------------------------------------------------------------
+constexpr int kRegsPerLane = kMaxCand / 32;
+
+__global__ void __launch_bounds__(256)
+topk_gate_kernel(const float *__restrict__ logits, int T, int n_real, int n_cand, int K, int gate_mode,
+                 int32_t *__restrict__ topk_idx, float *__restrict__ topk_w) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (t >= T) return;
+    float v[kRegsPerLane];
+    const float *row = logits + (size_t)t * n_cand;
+#pragma unroll
+    for (int r = 0; r < kRegsPerLane; ++r) {
+        const int j = r * 32 + lane;
+        v[r] = (j < n_cand) ? row[j] : -INFINITY;
+    }
+    // row maximum and softmax denominator over all candidates
+    float m = v[0];
+#pragma unroll
+    for (int r = 1; r < kRegsPerLane; ++r) m = fmaxf(m, v[r]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, o));
+    float den = 0.f;
+#pragma unroll
+    for (int r = 0; r < kRegsPerLane; ++r) {
+        const int j = r * 32 + lane;
+        if (j < n_cand) den += expf(v[r] - m);
+    }
+    den = warp_sum(den);
+
+    unsigned taken = 0;  // bit r set: this lane's register r was already selected
+    int my_idx = -1;     // lane k keeps slot k
+    float my_p = 0.f;
+    float sum_sel = 0.f, sum_real = 0.f;
+    for (int k = 0; k < K; ++k) {
+        float bv = -INFINITY;
+        int bj = 0x7fffffff;
+#pragma unroll
+        for (int r = 0; r < kRegsPerLane; ++r) {
+            const int j = r * 32 + lane;
+            if (j < n_cand && !((taken >> r) & 1u) && (v[r] > bv || bj == 0x7fffffff)) { bv = v[r]; bj = j; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(kFull, bv, o);
+            const int oj = __shfl_xor_sync(kFull, bj, o);
+            if (oj != 0x7fffffff && (bj == 0x7fffffff || ov > bv || (ov == bv && oj < bj))) { bv = ov; bj = oj; }
+        }
+        if ((bj & 31) == lane) taken |= 1u << (bj >> 5);
+        const float p = expf(bv - m) / den;
+        sum_sel += p;
+        if (bj < n_real) sum_real += p;
+        if (lane == k) { my_idx = bj; my_p = p; }
+    }
+    if (lane < K) {
+        float w = my_p;
+        if (gate_mode == ZEDA_GATE_TOPK_NORM) w = my_p / sum_sel;
+        else if (gate_mode == ZEDA_GATE_RENORM_REAL) w = (my_idx < n_real && sum_real > 0.f) ? my_p / sum_real : 0.f;
+        topk_idx[(size_t)t * K + lane] = my_idx;
+        topk_w[(size_t)t * K + lane] = w;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Counting sort, pass 1: per-CTA histogram of the normal-expert slots of kSortTokens tokens.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+slot_hist_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real,
+                 int32_t *__restrict__ block_hist) {
+    extern __shared__ int32_t hist[];  // [n_real]
+    for (int e = threadIdx.x; e < n_real; e += blockDim.x) hist[e] = 0;
+    __syncthreads();
+    const int s0 = blockIdx.x * kSortTokens * K;
+    const int s1 = min(T * K, s0 + kSortTokens * K);
+    for (int s = s0 + threadIdx.x; s < s1; s += blockDim.x) {
+        const int e = topk_idx[s];
+        if (e < n_real) atomicAdd(&hist[e], 1);
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < n_real; e += blockDim.x) block_hist[(size_t)blockIdx.x * n_real + e] = hist[e];
+}
+
+// ---------------------------------------------------------------------------------------------
+// Counting sort, pass 2 (one CTA): column-wise exclusive scan over the CTA histograms, expert
+// counts, exclusive offsets, P, U, and the work lists of the expert kernels.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(512)
+expert_scan_kernel(int32_t *__restrict__ block_hist, int nblk, int n_real, int total_slots,
+                   int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
+                   int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
+                   int32_t *__restrict__ chunk_expert, int32_t *__restrict__ chunk_row0,
+                   int32_t *__restrict__ tile_expert, int32_t *__restrict__ tile_row0) {
+    __shared__ int32_t s_cnt[kMaxCand];
+    __shared__ int32_t s_off[kMaxCand + 1];
+    __shared__ int32_t s_chunk[kMaxCand + 1];
+    __shared__ int32_t s_tile[kMaxCand + 1];
+    const int e = threadIdx.x;
+    if (e < n_real) {
+        int run = 0;
+        for (int b = 0; b < nblk; ++b) {
+            const int c = block_hist[(size_t)b * n_real + e];
+            block_hist[(size_t)b * n_real + e] = run;  // pairs of expert e in earlier CTAs
+            run += c;
+        }
+        s_cnt[e] = run;
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        // warp 0 scans the three per-expert sequences in chunks of 32
+        int base_off = 0, base_chunk = 0, base_tile = 0, active = 0, max_rows = 0;
+        for (int e0 = 0; e0 < n_real; e0 += 32) {
+            const int i = e0 + threadIdx.x;
+            const int c = (i < n_real) ? s_cnt[i] : 0;
+            const int ch = (c + kChunkRows - 1) / kChunkRows;
+            const int tl = (c + kTileM - 1) / kTileM;
+            int so = c, sc = ch, st = tl;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int a = __shfl_up_sync(kFull, so, o);
+                const int b = __shfl_up_sync(kFull, sc, o);
+                const int g = __shfl_up_sync(kFull, st, o);
+                if ((int)threadIdx.x >= o) { so += a; sc += b; st += g; }
+            }
+            if (i < n_real) {
+                s_off[i] = base_off + so - c;
+                s_chunk[i] = base_chunk + sc - ch;
+                s_tile[i] = base_tile + st - tl;
+            }
+            base_off += __shfl_sync(kFull, so, 31);
+            base_chunk += __shfl_sync(kFull, sc, 31);
+            base_tile += __shfl_sync(kFull, st, 31);
+            active += __popc(__ballot_sync(kFull, c > 0));
+            int mx = c;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(kFull, mx, o));
+            max_rows = max(max_rows, mx);
+        }
+        if (threadIdx.x == 0) {
+            s_off[n_real] = base_off;
+            s_chunk[n_real] = base_chunk;
+            s_tile[n_real] = base_tile;
+            meta[kMetaPairs] = base_off;
+            meta[kMetaActive] = active;
+            meta[kMetaZeroSlots] = total_slots - base_off;
+            meta[kMetaChunks] = base_chunk;
+            meta[kMetaTiles] = base_tile;
+            meta[kMetaMaxRows] = max_rows;
+            if (n_pairs_out) *n_pairs_out = base_off;
+        }
+    }
+    __syncthreads();
+    if (e < n_real) {
+        const int c = s_cnt[e];
+        if (counts) counts[e] = c;
+        offsets[e] = s_off[e];
+        int ci = s_chunk[e];
+        for (int r = 0; r < c; r += kChunkRows, ++ci) { chunk_expert[ci] = e; chunk_row0[ci] = r; }
+        int ti = s_tile[e];
+        for (int r = 0; r < c; r += kTileM, ++ti) { tile_expert[ti] = e; tile_row0[ti] = r; }
+    }
+    if (e == 0) offsets[n_real] = s_off[n_real];
+}
+
+// ---------------------------------------------------------------------------------------------
+// Counting sort, pass 3: stable placement.  Each CTA re-walks its kSortTokens*K slots in slot
+// order; each warp owns a contiguous run of slots, ranks equal experts inside a 32-slot step with
+// match.any / popc (a warp-level prefix count) and carries per-expert running positions in shared
+// memory.  No atomics decide a position, so the order is (expert, token) ascending every run.
+// ---------------------------------------------------------------------------------------------
+constexpr int kPlaceWarps = 8;
+
+__global__ void __launch_bounds__(kPlaceWarps * 32)
+slot_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real,
+                  const int32_t *__restrict__ block_base, const int32_t *__restrict__ offsets,
+                  int32_t *__restrict__ perm, int32_t *__restrict__ perm_user,
+                  int32_t *__restrict__ inv, int32_t *__restrict__ pair_token) {
+    extern __shared__ int32_t pos[];  // [kPlaceWarps][n_real]
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int i = threadIdx.x; i < kPlaceWarps * n_real; i += blockDim.x) pos[i] = 0;
+    __syncthreads();
+    const int s0 = blockIdx.x * kSortTokens * K;
+    const int s1 = min(T * K, s0 + kSortTokens * K);
+    const int per_warp = ((kSortTokens * K + kPlaceWarps - 1) / kPlaceWarps + 31) / 32 * 32;
+    const int w0 = s0 + warp * per_warp;
+    const int w1 = min(s1, w0 + per_warp);
+    int32_t *mine = pos + warp * n_real;
+    const unsigned lt = (1u << lane) - 1u;
+    // count this warp's slots per expert
+    for (int s = w0 + lane; s - lane < w1; s += 32) {
+        int e = (s < w1) ? topk_idx[s] : -1;
+        if (e >= n_real) e = -1;
+        const unsigned grp = __match_any_sync(kFull, e);
+        if (e >= 0 && (grp & lt) == 0) mine[e] += __popc(grp);
+        __syncwarp();
+    }
+    __syncthreads();
+    // turn counts into start positions: global offset + earlier CTAs + earlier warps
+    for (int e = threadIdx.x; e < n_real; e += blockDim.x) {
+        int run = offsets[e] + block_base[(size_t)blockIdx.x * n_real + e];
+        for (int w = 0; w < kPlaceWarps; ++w) {
+            const int c = pos[w * n_real + e];
+            pos[w * n_real + e] = run;
+            run += c;
+        }
+    }
+    __syncthreads();
+    for (int s = w0 + lane; s - lane < w1; s += 32) {
+        int e = (s < w1) ? topk_idx[s] : -1;
+        const bool in_range = s < w1;
+        if (e >= n_real) e = -1;
+        const unsigned grp = __match_any_sync(kFull, e);
+        int p = -1;
+        if (e >= 0) p = mine[e] + __popc(grp & lt);
+        __syncwarp();
+        if (e >= 0 && (grp & lt) == 0) mine[e] += __popc(grp);
+        __syncwarp();
+        if (in_range) {
+            inv[s] = p;
+            if (p >= 0) {
+                perm[p] = s;
+                if (perm_user) perm_user[p] = s;
+                pair_token[p] = s / K;
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Routing statistics (Eq. 4-6 forward values), two deterministic passes: per-CTA partial sums of
+// the selection indicator and of the softmax probabilities, then a fixed-order final reduction.
+// ---------------------------------------------------------------------------------------------
+constexpr int kStatTokens = 64;
+
+__global__ void __launch_bounds__(256)
+stats_partial_kernel(const float *__restrict__ logits, const int32_t *__restrict__ topk_idx, int T, int K,
+                     int n_cand, float *__restrict__ part) {
+    extern __shared__ float sm[];  // [2][n_cand]
+    float *sf = sm, *sp = sm + n_cand;
+    for (int i = threadIdx.x; i < 2 * n_cand; i += blockDim.x) sm[i] = 0.f;
+    __syncthreads();
+    __shared__ float s_max[kStatTokens], s_den[kStatTokens];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t0 = blockIdx.x * kStatTokens;
+    const int t1 = min(T, t0 + kStatTokens);
+    // per-token softmax maximum and denominator, one warp per token
+    for (int t = t0 + warp; t < t1; t += (blockDim.x >> 5)) {
+        const float *row = logits + (size_t)t * n_cand;
+        float m = -INFINITY;
+        for (int c = lane; c < n_cand; c += 32) m = fmaxf(m, row[c]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, o));
+        float den = 0.f;
+        for (int c = lane; c < n_cand; c += 32) den += expf(row[c] - m);
+        den = warp_sum(den);
+        if (lane == 0) { s_max[t - t0] = m; s_den[t - t0] = den; }
+    }
+    __syncthreads();
+    // one thread per candidate, tokens summed in increasing order
+    for (int j = threadIdx.x; j < n_cand; j += blockDim.x) {
+        float accp = 0.f, accf = 0.f;
+        for (int t = t0; t < t1; ++t) {
+            accp += expf(logits[(size_t)t * n_cand + j] - s_max[t - t0]) / s_den[t - t0];
+            for (int k = 0; k < K; ++k) accf += (topk_idx[(size_t)t * K + k] == j) ? 1.f : 0.f;
+        }
+        sf[j] = accf;
+        sp[j] = accp;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 2 * n_cand; i += blockDim.x) part[(size_t)blockIdx.x * 2 * n_cand + i] = sm[i];
+}
+
+__global__ void __launch_bounds__(512)
+stats_final_kernel(const float *__restrict__ part, int nblk, int T, int K, int n_real, int n_cand,
+                   float *__restrict__ f, float *__restrict__ p_mean, float *__restrict__ out) {
+    __shared__ float sf[kMaxCand], sp[kMaxCand];
+    const int j = threadIdx.x;
+    if (j < n_cand) {
+        float af = 0.f, ap = 0.f;
+        for (int b = 0; b < nblk; ++b) {
+            af += part[(size_t)b * 2 * n_cand + j];
+            ap += part[(size_t)b * 2 * n_cand + n_cand + j];
+        }
+        sf[j] = af / T;
+        sp[j] = ap / T;
+        if (f) f[j] = sf[j];
+        if (p_mean) p_mean[j] = sp[j];
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && out) {
+        float la = 0.f, fE = 0.f, pE = 0.f, fZ = 0.f, pZ = 0.f;
+        for (int i = 0; i < n_cand; ++i) {
+            la += sf[i] * sp[i];
+            if (i < n_real) { fE += sf[i]; pE += sp[i]; } else { fZ += sf[i]; pZ += sp[i]; }
+        }
+        out[0] = fZ / K;
+        out[1] = la;
+        out[2] = fE * pE;
+        out[3] = fZ * pZ;
+    }
+}
+
+}  // namespace
+
+int init_route_kernels(const zeda_moe *h) {
+    const size_t smem = (size_t)kTok * h->cfg.d_model * sizeof(__nv_bfloat16);
+    if (smem > 48 * 1024 &&
+        cudaFuncSetAttribute(router_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return -1;
+    return 0;
+}
+
+int launch_router_logits(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, cudaStream_t s) {
+    const int d = h->cfg.d_model, n_cand = h->cfg.n_real + h->cfg.n_zero;
+    const int tiles = (T + kTok - 1) / kTok;
+    // split the candidates over grid.y until the grid covers the SMs about twice
+    int splits = 1;
+    const int max_splits = (n_cand + 7) / 8;
+    while (tiles * splits < 2 * h->sm_count && splits < max_splits) splits *= 2;
+    if (splits > max_splits) splits = max_splits;
+    const int per = (n_cand + splits - 1) / splits;
+    const size_t smem = (size_t)kTok * d * sizeof(__nv_bfloat16);
+    router_logits_kernel<<<dim3(tiles, (n_cand + per - 1) / per), 256, smem, s>>>(
+        x, h->router_w, h->router_bias, T, d, n_cand, per, logits);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, const RouteOut &out, cudaStream_t s) {
+    const zeda_moe_config_t &c = h->cfg;
+    const int n_cand = c.n_real + c.n_zero, K = c.top_k;
+    const Workspace &ws = h->ws;
+    const int nblk = (T + kSortTokens - 1) / kSortTokens;
+    topk_gate_kernel<<<(T + 7) / 8, 256, 0, s>>>(logits, T, c.n_real, n_cand, K, c.gate_mode, ws.topk_idx, ws.topk_w);
+    slot_hist_kernel<<<nblk, 256, sizeof(int32_t) * c.n_real, s>>>(ws.topk_idx, T, K, c.n_real, ws.block_hist);
+    expert_scan_kernel<<<1, 512, 0, s>>>(ws.block_hist, nblk, c.n_real, T * K, ws.counts, ws.offsets, out.n_pairs,
+                                         ws.meta, ws.chunk_expert, ws.chunk_row0, ws.tile_expert, ws.tile_row0);
+    slot_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * kPlaceWarps * c.n_real, s>>>(
+        ws.topk_idx, T, K, c.n_real, ws.block_hist, ws.offsets, ws.perm, out.perm, ws.inv, ws.pair_token);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    // copies for a caller that asked for the routing itself
+    const cudaMemcpyKind d2d = cudaMemcpyDeviceToDevice;
+    if (out.topk_idx) cudaMemcpyAsync(out.topk_idx, ws.topk_idx, sizeof(int32_t) * (size_t)T * K, d2d, s);
+    if (out.topk_w) cudaMemcpyAsync(out.topk_w, ws.topk_w, sizeof(float) * (size_t)T * K, d2d, s);
+    if (out.counts) cudaMemcpyAsync(out.counts, ws.counts, sizeof(int32_t) * c.n_real, d2d, s);
+    if (out.offsets) cudaMemcpyAsync(out.offsets, ws.offsets, sizeof(int32_t) * (c.n_real + 1), d2d, s);
+    return cudaGetLastError() == cudaSuccess ? 4 : -1;
+}
+
+int launch_stats(const zeda_moe *h, const float *logits, const int32_t *topk_idx, int T, float *f,
+                 float *p_mean, float *out, cudaStream_t s) {
+    const zeda_moe_config_t &c = h->cfg;
+    const int n_cand = c.n_real + c.n_zero;
+    const int nblk = (T + kStatTokens - 1) / kStatTokens;
+    stats_partial_kernel<<<nblk, 256, sizeof(float) * 2 * n_cand, s>>>(logits, topk_idx, T, c.top_k, n_cand,
+                                                                      h->ws.stat_part);
+    stats_final_kernel<<<1, 512, 0, s>>>(h->ws.stat_part, nblk, T, c.top_k, c.n_real, n_cand, f, p_mean, out);
+    return cudaGetLastError() == cudaSuccess ? 2 : -1;
+}
+
+}  // namespace zeda

@@ -1,0 +1,354 @@
+// Host side of the C ABI: argument checks, workspace carving, stream-ordered launches.
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "zeda_internal.h"
+
+namespace zeda {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+}
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+bool config_ok(const zeda_moe_config_t *c, const char **why) {
+    const char *w = nullptr;
+    if (!c) w = "config is NULL";
+    else if (c->d_model < 64 || c->d_model % 64 || c->d_model > 8192) w = "d_model must be a multiple of 64 in [64, 8192]";
+    else if (c->d_expert < 64 || c->d_expert % 64 || c->d_expert > 8192) w = "d_expert must be a multiple of 64 in [64, 8192]";
+    else if (c->n_real < 1) w = "n_real must be >= 1";
+    else if (c->n_zero < 0) w = "n_zero must be >= 0";
+    else if (c->n_real + c->n_zero > kMaxCand) w = "n_real + n_zero must be <= 512";
+    else if (c->top_k < 1 || c->top_k > kMaxTopK) w = "top_k must be in [1, 16]";
+    else if (c->top_k > c->n_real + c->n_zero) w = "top_k exceeds the number of candidates";
+    else if (c->max_tokens < 1) w = "max_tokens must be >= 1";
+    else if ((long long)c->max_tokens * c->top_k >= (1LL << 27)) w = "max_tokens * top_k must be < 2^27";
+    else if (c->gate_mode < 0 || c->gate_mode > 2) w = "unknown gate_mode";
+    else if (c->expert_kind < 0 || c->expert_kind > 1) w = "unknown expert_kind";
+    else if ((c->flags & ZEDA_FLAG_FORCE_STREAM_EXPERTS) && (c->flags & ZEDA_FLAG_FORCE_TILE_EXPERTS)) w = "contradictory flags";
+    if (why) *why = w;
+    return w == nullptr;
+}
+
+// Walks the workspace layout; with base == nullptr it only measures.
+size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int *max_chunks, int *max_tiles) {
+    size_t off = 0;
+    auto take = [&](size_t bytes) -> void * {
+        void *p = base ? base + off : nullptr;
+        off = align_up(off + bytes, 256);
+        return p;
+    };
+    const size_t slots = (size_t)c.max_tokens * c.top_k;
+    const size_t n_cand = (size_t)c.n_real + c.n_zero;
+    const size_t nblk = (c.max_tokens + kSortTokens - 1) / kSortTokens;
+    const size_t chunks = slots / kChunkRows + c.n_real + 1;
+    const size_t tiles = slots / kTileM + c.n_real + 1;
+    const size_t nblk_stats = (c.max_tokens + 63) / 64;
+    Workspace w;
+    w.topk_idx = (int32_t *)take(slots * 4);
+    w.topk_w = (float *)take(slots * 4);
+    w.inv = (int32_t *)take(slots * 4);
+    w.perm = (int32_t *)take(slots * 4);
+    w.pair_token = (int32_t *)take(slots * 4);
+    w.block_hist = (int32_t *)take(nblk * c.n_real * 4);
+    w.counts = (int32_t *)take((size_t)c.n_real * 4);
+    w.offsets = (int32_t *)take((size_t)(c.n_real + 1) * 4);
+    w.meta = (int32_t *)take(kMetaCount * 4);
+    w.chunk_expert = (int32_t *)take(chunks * 4);
+    w.chunk_row0 = (int32_t *)take(chunks * 4);
+    w.tile_expert = (int32_t *)take(tiles * 4);
+    w.tile_row0 = (int32_t *)take(tiles * 4);
+    w.logits = (float *)take((size_t)c.max_tokens * n_cand * 4);
+    w.stat_part = (float *)take(nblk_stats * 2 * n_cand * 4);
+    // pair buffers carry kTileM rows of slack so that a full tile may be stored past the last pair
+    w.hmid = (__nv_bfloat16 *)take((slots + kTileM) * c.d_expert * 2);
+    w.obuf = (__nv_bfloat16 *)take((slots + kTileM) * c.d_model * 2);
+    w.x_stage = (__nv_bfloat16 *)take((size_t)c.max_tokens * c.d_model * 2);
+    w.y_stage = (__nv_bfloat16 *)take((size_t)c.max_tokens * c.d_model * 2);
+    if (ws) *ws = w;
+    if (max_chunks) *max_chunks = (int)chunks;
+    if (max_tiles) *max_tiles = (int)tiles;
+    return off;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+zeda_status_t cuda_fail(const char *what, cudaError_t e) {
+    set_error("%s: %s", what, cudaGetErrorString(e));
+    return ZEDA_ERR_CUDA;
+}
+
+zeda_status_t check_call(zeda_moe_t *h, const void *in, int32_t T, const char *in_name) {
+    if (!h) { set_error("handle is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    if (T < 0 || T > h->cfg.max_tokens) { set_error("T=%d outside [0, max_tokens=%d]", T, h->cfg.max_tokens); return ZEDA_ERR_INVALID_ARG; }
+    if (T > 0 && !in) { set_error("%s is NULL", in_name); return ZEDA_ERR_INVALID_ARG; }
+    if (T > 0 && !aligned16(in)) { set_error("%s is not 16-byte aligned", in_name); return ZEDA_ERR_INVALID_ARG; }
+    cudaError_t e = cudaSetDevice(h->cfg.device);
+    if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
+    return ZEDA_OK;
+}
+
+// Routing into the workspace (+ optional user copies); returns launches or <0.
+int route_into(zeda_moe_t *h, const __nv_bfloat16 *x, const float *logits_in, int T, const RouteOut &out, cudaStream_t s) {
+    int n = 0;
+    const float *logits = logits_in;
+    if (!logits) {
+        int r = launch_router_logits(h, x, T, h->ws.logits, s);
+        if (r < 0) return r;
+        n += r;
+        logits = h->ws.logits;
+    }
+    int r = launch_route_from_logits(h, logits, T, out, s);
+    if (r < 0) return r;
+    return n + r;
+}
+
+zeda_status_t forward_device(zeda_moe_t *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s) {
+    const bool prof = h->profiling;
+    auto mark = [&](int i) { if (prof) cudaEventRecord(h->ev[i], s); };
+    mark(0);
+    int n = launch_router_logits(h, x, T, h->ws.logits, s);
+    if (n < 0) return cuda_fail("router launch", cudaGetLastError());
+    mark(1);
+    RouteOut none = {};
+    int r = launch_route_from_logits(h, h->ws.logits, T, none, s);
+    if (r < 0) return cuda_fail("routing launch", cudaGetLastError());
+    n += r;
+    mark(2);
+    r = launch_experts_gemm1(h, x, T, s);
+    if (r < 0) return cuda_fail("expert GEMM1 launch", cudaGetLastError());
+    n += r;
+    mark(3);
+    r = launch_experts_gemm2(h, T, s);
+    if (r < 0) return cuda_fail("expert GEMM2 launch", cudaGetLastError());
+    n += r;
+    mark(4);
+    r = launch_combine(h, x, T, y, s);
+    if (r < 0) return cuda_fail("combine launch", cudaGetLastError());
+    mark(5);
+    h->profiled_last = prof;
+    h->last_launches = n + r;
+    return ZEDA_OK;
+}
+
+}  // namespace
+}  // namespace zeda
+
+using namespace zeda;
+
+extern "C" {
+
+size_t zeda_moe_workspace_bytes(const zeda_moe_config_t *cfg) {
+    const char *why = nullptr;
+    if (!config_ok(cfg, &why)) { set_error("%s", why); return 0; }
+    return carve(*cfg, nullptr, nullptr, nullptr, nullptr);
+}
+
+zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_w, const float *router_bias,
+                              const void *w_gate_up, const void *w_down, void *workspace, size_t workspace_bytes,
+                              zeda_moe_t **out) {
+    if (out) *out = nullptr;
+    const char *why = nullptr;
+    if (!config_ok(cfg, &why)) {
+        set_error("%s", why);
+        const bool shape = cfg && why && (strstr(why, "multiple of 64") || strstr(why, "<= 512") || strstr(why, "[1, 16]"));
+        return shape ? ZEDA_ERR_UNSUPPORTED : ZEDA_ERR_INVALID_ARG;
+    }
+    if (!out) { set_error("out is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    if (!router_w || !w_gate_up || !w_down || !workspace) { set_error("a required pointer is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    if (!aligned16(router_w) || !aligned16(w_gate_up) || !aligned16(w_down) || (router_bias && (reinterpret_cast<uintptr_t>(router_bias) & 3u))) {
+        set_error("weights must be 16-byte aligned");
+        return ZEDA_ERR_INVALID_ARG;
+    }
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) { set_error("workspace must be 256-byte aligned"); return ZEDA_ERR_INVALID_ARG; }
+    const size_t need = carve(*cfg, nullptr, nullptr, nullptr, nullptr);
+    if (workspace_bytes < need) { set_error("workspace has %zu bytes, %zu needed", workspace_bytes, need); return ZEDA_ERR_WORKSPACE; }
+    int ndev = 0;
+    cudaError_t e = cudaGetDeviceCount(&ndev);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDeviceCount", e);
+    if (cfg->device < 0 || cfg->device >= ndev) { set_error("device %d not present (%d devices)", cfg->device, ndev); return ZEDA_ERR_INVALID_ARG; }
+    e = cudaSetDevice(cfg->device);
+    if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, cfg->device);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDeviceProperties", e);
+    if (prop.major != 10) { set_error("this library is built for sm_100a only; device is sm_%d%d", prop.major, prop.minor); return ZEDA_ERR_UNSUPPORTED; }
+
+    zeda_moe *h = new (std::nothrow) zeda_moe();
+    if (!h) { set_error("out of host memory"); return ZEDA_ERR_INVALID_ARG; }
+    h->cfg = *cfg;
+    h->router_w = router_w;
+    h->router_bias = router_bias;
+    h->w_gate_up = static_cast<const __nv_bfloat16 *>(w_gate_up);
+    h->w_down = static_cast<const __nv_bfloat16 *>(w_down);
+    h->sm_count = prop.multiProcessorCount;
+    h->last_launches = 0;
+    h->tmaps = nullptr;
+    h->profiling = false;
+    h->profiled_last = false;
+    for (auto &ev : h->ev) ev = nullptr;
+    carve(*cfg, static_cast<unsigned char *>(workspace), &h->ws, &h->max_chunks, &h->max_tiles);
+    if (init_route_kernels(h) < 0) { delete h; return cuda_fail("kernel set-up", cudaGetLastError()); }
+    e = cudaMemset(h->ws.meta, 0, kMetaCount * 4);
+    if (e != cudaSuccess) { delete h; return cuda_fail("cudaMemset(meta)", e); }
+    e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { delete h; return cuda_fail("cudaDeviceSynchronize", e); }
+    *out = h;
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_route(zeda_moe_t *h, const void *x, int32_t T, int32_t *topk_idx, float *topk_w,
+                         int32_t *expert_counts, int32_t *expert_offsets, int32_t *perm, int32_t *n_pairs,
+                         void *stream) {
+    zeda_status_t st = check_call(h, x, T, "x");
+    if (st != ZEDA_OK || T == 0) return st;
+    RouteOut out = {topk_idx, topk_w, expert_counts, expert_offsets, perm, n_pairs};
+    int n = route_into(h, static_cast<const __nv_bfloat16 *>(x), nullptr, T, out, static_cast<cudaStream_t>(stream));
+    if (n < 0) return cuda_fail("routing launch", cudaGetLastError());
+    h->last_launches = n;
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_route_from_logits(zeda_moe_t *h, const float *logits, int32_t T, int32_t *topk_idx, float *topk_w,
+                                     int32_t *expert_counts, int32_t *expert_offsets, int32_t *perm,
+                                     int32_t *n_pairs, void *stream) {
+    zeda_status_t st = check_call(h, logits, T, "logits");
+    if (st != ZEDA_OK || T == 0) return st;
+    RouteOut out = {topk_idx, topk_w, expert_counts, expert_offsets, perm, n_pairs};
+    int n = route_into(h, nullptr, logits, T, out, static_cast<cudaStream_t>(stream));
+    if (n < 0) return cuda_fail("routing launch", cudaGetLastError());
+    h->last_launches = n;
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_router_logits(zeda_moe_t *h, const void *x, int32_t T, float *logits, void *stream) {
+    zeda_status_t st = check_call(h, x, T, "x");
+    if (st != ZEDA_OK || T == 0) return st;
+    if (!logits) { set_error("logits is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    int n = launch_router_logits(h, static_cast<const __nv_bfloat16 *>(x), T, logits, static_cast<cudaStream_t>(stream));
+    if (n < 0) return cuda_fail("router launch", cudaGetLastError());
+    h->last_launches = n;
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_moe_forward(zeda_moe_t *h, const void *x, int32_t T, void *y, void *stream) {
+    zeda_status_t st = check_call(h, x, T, "x");
+    if (st != ZEDA_OK || T == 0) return st;
+    if (!y || !aligned16(y)) { set_error("y is NULL or not 16-byte aligned"); return ZEDA_ERR_INVALID_ARG; }
+    const size_t bytes = (size_t)T * h->cfg.d_model * 2;
+    const char *xb = static_cast<const char *>(x), *yb = static_cast<const char *>(y);
+    if (xb < yb + bytes && yb < xb + bytes) { set_error("x and y overlap"); return ZEDA_ERR_INVALID_ARG; }
+    return forward_device(h, static_cast<const __nv_bfloat16 *>(x), T, static_cast<__nv_bfloat16 *>(y),
+                          static_cast<cudaStream_t>(stream));
+}
+
+zeda_status_t zeda_moe_forward_host(zeda_moe_t *h, const void *x_host, int32_t T, void *y_host, void *stream) {
+    if (!h) { set_error("handle is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    if (T < 0 || T > h->cfg.max_tokens) { set_error("T=%d outside [0, max_tokens=%d]", T, h->cfg.max_tokens); return ZEDA_ERR_INVALID_ARG; }
+    if (T == 0) return ZEDA_OK;
+    if (!x_host || !y_host) { set_error("host buffer is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    cudaError_t e = cudaSetDevice(h->cfg.device);
+    if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t bytes = (size_t)T * h->cfg.d_model * 2;
+    e = cudaMemcpyAsync(h->ws.x_stage, x_host, bytes, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail("copy of x to the device", e);
+    zeda_status_t st = forward_device(h, h->ws.x_stage, T, h->ws.y_stage, s);
+    if (st != ZEDA_OK) return st;
+    e = cudaMemcpyAsync(y_host, h->ws.y_stage, bytes, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail("copy of y to the host", e);
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_moe_stats(zeda_moe_t *h, const void *x, int32_t T, float *f, float *p_mean, float *out, void *stream) {
+    zeda_status_t st = check_call(h, x, T, "x");
+    if (st != ZEDA_OK || T == 0) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    RouteOut none = {};
+    int n = route_into(h, static_cast<const __nv_bfloat16 *>(x), nullptr, T, none, s);
+    if (n < 0) return cuda_fail("routing launch", cudaGetLastError());
+    int r = launch_stats(h, h->ws.logits, h->ws.topk_idx, T, f, p_mean, out, s);
+    if (r < 0) return cuda_fail("stats launch", cudaGetLastError());
+    h->last_launches = n + r;
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_moe_last_counters(zeda_moe_t *h, int64_t out[4], void *stream) {
+    if (!h || !out) { set_error("NULL argument"); return ZEDA_ERR_INVALID_ARG; }
+    cudaError_t e = cudaSetDevice(h->cfg.device);
+    if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
+    int32_t meta[kMetaCount];
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    e = cudaMemcpyAsync(meta, h->ws.meta, sizeof meta, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail("cudaMemcpyAsync(meta)", e);
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
+    out[0] = meta[kMetaPairs];
+    out[1] = meta[kMetaActive];
+    out[2] = meta[kMetaZeroSlots];
+    out[3] = h->last_launches;
+    if (meta[kMetaError] != 0) { set_error("a bounded device wait expired (code %d)", meta[kMetaError]); return ZEDA_ERR_TIMEOUT; }
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_moe_set_profiling(zeda_moe_t *h, int32_t enable) {
+    if (!h) { set_error("handle is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    cudaError_t e = cudaSetDevice(h->cfg.device);
+    if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
+    if (enable && !h->ev[0]) {
+        for (auto &ev : h->ev) {
+            e = cudaEventCreate(&ev);
+            if (e != cudaSuccess) return cuda_fail("cudaEventCreate", e);
+        }
+    }
+    h->profiling = enable != 0;
+    if (!enable) h->profiled_last = false;
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_moe_stage_ms(zeda_moe_t *h, float ms[ZEDA_STAGE_COUNT]) {
+    if (!h || !ms) { set_error("NULL argument"); return ZEDA_ERR_INVALID_ARG; }
+    if (!h->profiled_last) { set_error("the last forward call was not profiled"); return ZEDA_ERR_INVALID_ARG; }
+    cudaError_t e = cudaEventSynchronize(h->ev[ZEDA_STAGE_COUNT]);
+    if (e != cudaSuccess) return cuda_fail("cudaEventSynchronize", e);
+    for (int i = 0; i < ZEDA_STAGE_COUNT; ++i) {
+        e = cudaEventElapsedTime(&ms[i], h->ev[i], h->ev[i + 1]);
+        if (e != cudaSuccess) return cuda_fail("cudaEventElapsedTime", e);
+    }
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_moe_destroy(zeda_moe_t *h) {
+    if (!h) return ZEDA_OK;
+    zeda_status_t st = ZEDA_OK;
+    if (cudaSetDevice(h->cfg.device) == cudaSuccess) {
+        int32_t err = 0;
+        cudaError_t e = cudaDeviceSynchronize();
+        if (e == cudaSuccess) e = cudaMemcpy(&err, h->ws.meta + kMetaError, 4, cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) st = cuda_fail("zeda_moe_destroy", e);
+        else if (err != 0) { set_error("a bounded device wait expired (code %d)", err); st = ZEDA_ERR_TIMEOUT; }
+    }
+    for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
+    if (h->tmaps) free(h->tmaps);
+    delete h;
+    return st;
+}
+
+const char *zeda_last_error(void) { return g_err; }
+
+const char *zeda_version(void) { return "zeda-moe 0.1 (sm_100a)"; }
+
+}  // extern "C"

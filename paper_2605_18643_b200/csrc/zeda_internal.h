@@ -1,0 +1,94 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "zeda.h"
+
+namespace zeda {
+
+constexpr int kMaxCand = 512;       // N + N_Z limit (16 logits per lane in the top-K warp)
+constexpr int kMaxTopK = 16;
+constexpr int kSortTokens = 128;    // tokens per CTA in the counting sort (histogram / placement)
+constexpr int kChunkRows = 32;      // pair rows per work chunk of the streaming expert kernels
+constexpr int kTileM = 128;         // pair rows per tile of the tcgen05 expert kernels
+
+// Device-resident counters of one call.
+enum MetaSlot {
+    kMetaPairs = 0,      // P
+    kMetaActive = 1,     // U
+    kMetaZeroSlots = 2,  // slots that landed on zero experts
+    kMetaChunks = 3,     // work chunks for the streaming kernels
+    kMetaTiles = 4,      // M tiles for the tile kernels
+    kMetaError = 5,      // sticky error word written by bounded device waits
+    kMetaMaxRows = 6,    // largest per-expert pair count
+    kMetaCount = 16
+};
+
+struct Workspace {
+    int32_t *topk_idx;     // [maxT*K]
+    float *topk_w;         // [maxT*K]
+    int32_t *inv;          // [maxT*K] slot -> sorted position, -1 for zero slots
+    int32_t *perm;         // [maxT*K] sorted position -> slot
+    int32_t *pair_token;   // [maxT*K] sorted position -> token
+    int32_t *block_hist;   // [nblk*N]
+    int32_t *counts;       // [N]
+    int32_t *offsets;      // [N+1]
+    int32_t *meta;         // [kMetaCount]
+    int32_t *chunk_expert; // [maxChunks]
+    int32_t *chunk_row0;   // [maxChunks]
+    int32_t *tile_expert;  // [maxTiles]
+    int32_t *tile_row0;    // [maxTiles]
+    float *logits;         // [maxT*(N+N_Z)]
+    float *stat_part;      // [nblk_stats * 2 * (N+N_Z)]
+    __nv_bfloat16 *hmid;   // [maxT*K, He]
+    __nv_bfloat16 *obuf;   // [maxT*K, d]
+    __nv_bfloat16 *x_stage;// [maxT, d]
+    __nv_bfloat16 *y_stage;// [maxT, d]
+};
+
+struct RouteOut {  // where one routing pass writes (user buffers or workspace)
+    int32_t *topk_idx;
+    float *topk_w;
+    int32_t *counts;
+    int32_t *offsets;
+    int32_t *perm;
+    int32_t *n_pairs;  // optional extra copy of P
+};
+
+}  // namespace zeda
+
+struct zeda_moe {
+    zeda_moe_config_t cfg;
+    const float *router_w;
+    const float *router_bias;
+    const __nv_bfloat16 *w_gate_up;
+    const __nv_bfloat16 *w_down;
+    zeda::Workspace ws;
+    int sm_count;
+    int max_chunks;
+    int max_tiles;
+    int last_launches;
+    void *tmaps;  // host-side tensor maps of the tile path (owned)
+    bool profiling;
+    bool profiled_last;
+    cudaEvent_t ev[ZEDA_STAGE_COUNT + 1];
+};
+
+namespace zeda {
+
+// ---- launchers (each returns the number of kernels it enqueued, or <0 on a launch error) ----
+int init_route_kernels(const zeda_moe *h);
+int launch_router_logits(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, cudaStream_t s);
+int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, const RouteOut &out, cudaStream_t s);
+int launch_stats(const zeda_moe *h, const float *logits, const int32_t *topk_idx, int T, float *f,
+                 float *p_mean, float *out, cudaStream_t s);
+int launch_experts_gemm1(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
+int launch_experts_gemm2(const zeda_moe *h, int T, cudaStream_t s);
+int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s);
+
+void set_error(const char *fmt, ...);
+
+}  // namespace zeda

@@ -242,3 +242,18 @@ def rmsnorm_bf16(r: torch.Tensor, eps: float = 1e-6) -> torch.Tensor:
     of the paper's method): fp32 math, bf16 result."""
     rf = r.float()
     return (rf * torch.rsqrt(rf.pow(2).mean(dim=-1, keepdim=True) + eps)).to(torch.bfloat16)
+
+
+def replica_tokens(wl: Workload, rank: int) -> torch.Tensor:
+    """A fresh token batch for data-parallel replica `rank` of the same layer: x ~ N(0,1) from a
+    rank-derived seed, rows redrawn until the layer's router sees the top-K tie margin."""
+    x = _normal((wl.T, wl.d), 1.0, 5000 + rank, _ID_X, torch.bfloat16)
+    margin = TIE_MARGIN * _MARGIN_SLACK
+    for attempt in range(1, 64):
+        gaps = _topk_gaps(_logits32(x, wl.router_w, wl.router_bias), wl.K)
+        bad = torch.nonzero(gaps < margin).flatten()
+        if bad.numel() == 0:
+            return x
+        g = _gen(5000 + rank, _ID_REDRAW, attempt)
+        x[bad] = torch.randn(bad.numel(), wl.d, generator=g, dtype=torch.float32).to(torch.bfloat16)
+    raise RuntimeError("could not reach the top-K tie margin")

@@ -1,0 +1,265 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle on the same seeded inputs.
+
+Bars: routing indices, per-expert counts, offsets, permutation and P bit-exact; routing weights
+within fp32 rounding (rel 1e-5); layer output rel-L2 <= 1e-2 and max-abs <= 5e-2 * RMS(y).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_18643_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+REL_L2 = 1e-2
+MAX_ABS_RMS = 5e-2
+W_RTOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def zeda():
+    from paper_2605_18643_b200 import zeda as z
+    return z
+
+
+def np_bias(wl):
+    return None if wl.router_bias is None else wl.router_bias.numpy()
+
+
+def oracle_route(wl, gate_mode=0):
+    l = oracle.logits(inputs.bits(wl.x), wl.router_w.numpy(), np_bias(wl))
+    idx, w = oracle.route(l, wl.E, wl.Z, wl.K, gate_mode)
+    counts, offsets, perm, P = oracle.compact(idx, wl.E)
+    return l, idx, w, counts, offsets, perm, P
+
+
+def oracle_forward(wl, token_ids=None, gate_mode=0, expert_kind=0):
+    return oracle.forward(inputs.bits(wl.x), wl.router_w.numpy(), np_bias(wl), inputs.bits(wl.w_gate_up),
+                          inputs.bits(wl.w_down), wl.E, wl.Z, wl.K, gate_mode=gate_mode,
+                          expert_kind=expert_kind, token_ids=token_ids)
+
+
+def check_route(o, idx, w, counts, offsets, perm, P):
+    assert np.array_equal(o["topk_idx"].cpu().numpy(), idx)
+    assert int(o["n_pairs"].item()) == P
+    assert np.array_equal(o["counts"].cpu().numpy(), counts)
+    assert np.array_equal(o["offsets"].cpu().numpy(), offsets)
+    got_perm = o["perm"].cpu().numpy()
+    assert np.array_equal(got_perm[:P], perm)
+    assert np.all(got_perm[P:] == -1)                       # the tail is left untouched
+    gw = o["topk_w"].cpu().numpy().astype(np.float64)
+    assert np.allclose(gw, w, rtol=W_RTOL, atol=1e-30)
+
+
+def check_y(y_gpu, y_ref):
+    y_gpu = y_gpu.float().cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(y_gpu))
+    num = np.linalg.norm(y_gpu - y_ref)
+    den = np.linalg.norm(y_ref)
+    rms = np.sqrt(np.mean(y_ref ** 2))
+    if den == 0.0:
+        assert num == 0.0
+        return 0.0
+    assert num / den <= REL_L2, "rel L2 %.3e" % (num / den)
+    assert np.max(np.abs(y_gpu - y_ref)) <= MAX_ABS_RMS * rms
+    return num / den
+
+
+def run_layer(zeda, wl, token_ids=None, gate_mode=0, expert_kind=0, flags=0, check_routing=True):
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev, gate_mode=gate_mode, expert_kind=expert_kind, flags=flags)
+    x = wl.x.to(dev)
+    if check_routing:
+        l, idx, w, counts, offsets, perm, P = oracle_route(wl, gate_mode)
+        gl = m.router_logits(x).cpu().numpy()
+        assert np.max(np.abs(gl.astype(np.float64) - l.astype(np.float64))) < 2e-5
+        check_route(m.route(x), idx, w, counts, offsets, perm, P)
+    y = m.forward(x)
+    torch.cuda.synchronize()
+    y_ref, idx_ref, _ = oracle_forward(wl, token_ids, gate_mode, expert_kind)
+    ysel = y if token_ids is None else y[torch.as_tensor(token_ids, device=dev, dtype=torch.long)]
+    err = check_y(ysel, y_ref)
+    # tokens without a surviving slot: every element is +0 (bit pattern 0)
+    if expert_kind == 0:
+        dead = np.nonzero((idx_ref >= wl.E).all(axis=1))[0]
+        if dead.size:
+            rows = ysel[torch.as_tensor(dead, device=dev, dtype=torch.long)].view(torch.int16)
+            assert int(rows.abs().max().item()) == 0
+    P_dev, U_dev, zero_slots, launches = m.last_counters()
+    assert launches > 0
+    m.close()
+    return err, (P_dev, U_dev, zero_slots)
+
+
+# ---------------------------------------------------------------------------------- tiny layer
+
+def test_tiny_routing_and_forward(zeda):
+    wl = inputs.tiny()
+    err, (P, U, zs) = run_layer(zeda, wl)
+    assert P + zs == wl.T * wl.K and 0 < P < wl.T * wl.K
+
+
+@pytest.mark.parametrize("gate_mode", [0, 1, 2])
+@pytest.mark.parametrize("expert_kind", [0, 1])
+def test_tiny_gate_modes_and_copy_experts(zeda, gate_mode, expert_kind):
+    run_layer(zeda, inputs.tiny(seed=1), gate_mode=gate_mode, expert_kind=expert_kind)
+
+
+def test_tiny_static_layer_z0(zeda):
+    wl = inputs.tiny(seed=2, Z=0, zero_fraction=None)
+    err, (P, U, zs) = run_layer(zeda, wl)
+    assert zs == 0 and P == wl.T * wl.K
+
+
+def test_route_from_logits_is_bit_exact_with_ties(zeda):
+    wl = inputs.tiny()
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev, max_tokens=300)
+    rng = np.random.default_rng(0)
+    l = rng.standard_normal((300, wl.E + wl.Z)).astype(np.float32)
+    l[:50] = np.round(l[:50] * 2) / 2          # many exact ties
+    l[50] = 0.0
+    idx, w = oracle.route(l, wl.E, wl.Z, wl.K)
+    counts, offsets, perm, P = oracle.compact(idx, wl.E)
+    o = m.route_from_logits(torch.from_numpy(l).to(dev))
+    torch.cuda.synchronize()
+    check_route(o, idx, w, counts, offsets, perm, P)
+    m.close()
+
+
+def test_forward_is_deterministic(zeda):
+    wl = inputs.tiny(seed=4)
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev)
+    x = wl.x.to(dev)
+    a = m.forward(x).clone()
+    b = m.forward(x).clone()
+    torch.cuda.synchronize()
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    m.close()
+
+
+# ---------------------------------------------------------------------------------- edge cases
+
+@pytest.mark.parametrize("T", [1, 7, 129, 257])
+def test_ragged_token_counts(zeda, T):
+    run_layer(zeda, inputs.tiny(seed=5, T=T))
+
+
+def test_empty_batch_touches_nothing(zeda):
+    wl = inputs.tiny()
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev)
+    x = torch.empty((0, wl.d), dtype=torch.bfloat16, device=dev)
+    y = m.forward(x)
+    assert y.shape == (0, wl.d)
+    m.close()
+
+
+def test_every_slot_on_a_zero_expert(zeda):
+    wl = inputs.tiny(seed=6)
+    wl.router_bias[wl.E:] += 50.0
+    err, (P, U, zs) = run_layer(zeda, wl)
+    assert P == 0 and U == 0 and zs == wl.T * wl.K
+
+
+def test_all_tokens_on_one_expert(zeda):
+    wl = inputs.tiny(seed=7, T=200)
+    wl.router_bias[:wl.E] -= 50.0
+    wl.router_bias[3] += 100.0
+    err, (P, U, zs) = run_layer(zeda, wl)
+    o = oracle_route(wl)
+    assert o[3][3] == wl.T and (np.delete(o[3], 3) == 0).all() and U == 1   # expert 3 has every token
+
+
+def test_argument_errors(zeda):
+    wl = inputs.tiny()
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev)
+    x = wl.x.to(dev)
+    with pytest.raises(zeda.ZedaError) as e:
+        m.forward(torch.cat([x, x]))                        # T > max_tokens
+    assert e.value.status == zeda.ERR_INVALID_ARG
+    st = zeda.lib.zeda_moe_forward(m._h, x.data_ptr() + 2, wl.T - 1, x.data_ptr(), None)
+    assert st == zeda.ERR_INVALID_ARG                       # misaligned
+    st = zeda.lib.zeda_moe_forward(m._h, x.data_ptr(), wl.T, x.data_ptr(), None)
+    assert st == zeda.ERR_INVALID_ARG                       # x and y overlap
+    y = m.forward(x)                                        # the handle still works afterwards
+    torch.cuda.synchronize()
+    assert torch.isfinite(y.float()).all()
+    m.close()
+
+
+def test_host_buffer_entry_point(zeda):
+    wl = inputs.tiny(seed=8)
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev)
+    y_dev = m.forward(wl.x.to(dev)).cpu()
+    y_host = m.forward_host(wl.x.pin_memory())
+    assert torch.equal(y_dev.view(torch.int16), y_host.view(torch.int16))
+    y_pageable = m.forward_host(wl.x.clone())
+    assert torch.equal(y_dev.view(torch.int16), y_pageable.view(torch.int16))
+    m.close()
+
+
+def test_routing_statistics(zeda):
+    wl = inputs.tiny(seed=9, T=200)
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev)
+    f, p, o = m.stats(wl.x.to(dev))
+    l, idx, *_ = oracle_route(wl)
+    s = oracle.stats(l, idx, wl.E, wl.Z, alpha=1.0, group_w=1.0)
+    assert np.allclose(f.cpu().numpy(), s["f"], rtol=1e-5, atol=1e-7)
+    assert np.allclose(p.cpu().numpy(), s["P"], rtol=1e-4, atol=1e-7)
+    o = o.cpu().numpy().astype(np.float64)
+    assert np.isclose(o[0], s["r_ze"], rtol=1e-5)
+    n = wl.E + wl.Z
+    assert np.isclose(o[1] * n / wl.K, s["L_A"], rtol=1e-4)
+    assert np.isclose((wl.E + wl.Z) / wl.K * (o[2] / wl.E + o[3] / wl.Z), s["L_GA"], rtol=1e-4)
+    m.close()
+
+
+# ---------------------------------------------------------------------------------- full-size configs
+
+def test_decode_config_full_parity(zeda):
+    wl = inputs.decode()
+    err, (P, U, zs) = run_layer(zeda, wl)
+    assert abs(zs / (wl.T * wl.K) - 0.5) < 0.03
+
+
+def test_decode_config_static_reference(zeda):
+    wl = inputs.decode(Z=0, zero_fraction=None, token_shift=0.0)
+    run_layer(zeda, wl)
+
+
+def sample_tokens(T, n, seed):
+    return np.sort(np.random.default_rng(seed).choice(T, size=n, replace=False)).astype(np.int32)
+
+
+def test_prefill_config_routing_exact_and_sampled_outputs(zeda):
+    wl = inputs.prefill()
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev)
+    x = wl.x.to(dev)
+    # routing of all 8192 tokens, bit-exact (oracle routing only: no expert math)
+    _, idx, w = oracle.forward(inputs.bits(wl.x), wl.router_w.numpy(), np_bias(wl), inputs.bits(wl.w_gate_up),
+                               inputs.bits(wl.w_down), wl.E, wl.Z, wl.K, want_y=False)
+    counts, offsets, perm, P = oracle.compact(idx, wl.E)
+    check_route(m.route(x), idx, w, counts, offsets, perm, P)
+    assert counts.max() > 10 * max(1, counts.min())        # the Zipf skew is there
+    # outputs on a token sample (each token's output depends on its own row only)
+    ids = sample_tokens(wl.T, 192, 0)
+    y = m.forward(x)
+    torch.cuda.synchronize()
+    y_ref, _, _ = oracle_forward(wl, ids)
+    check_y(y[torch.as_tensor(ids, device=dev, dtype=torch.long)], y_ref)
+    m.close()
+
+
+@pytest.mark.parametrize("f", [0.0, 0.25, 0.5, 0.75])
+def test_sweep_config_sampled(zeda, f):
+    wl = inputs.sweep_point(f)
+    ids = sample_tokens(wl.T, 64, int(f * 100))
+    err, (P, U, zs) = run_layer(zeda, wl, token_ids=ids, check_routing=False)
+    assert abs(zs / (wl.T * wl.K) - f) < 0.02
