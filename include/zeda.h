@@ -159,6 +159,38 @@ enum { ZEDA_STAGE_ROUTER = 0, ZEDA_STAGE_SORT = 1, ZEDA_STAGE_GEMM1 = 2, ZEDA_ST
 zeda_status_t zeda_moe_set_profiling(zeda_moe_t *h, int32_t enable);
 zeda_status_t zeda_moe_stage_ms(zeda_moe_t *h, float ms[ZEDA_STAGE_COUNT]);
 
+/* Compaction and counting sort without any device allocation.  (The paper has no counterpart of
+ * this entry point; it exists for the callers described here.)
+ *
+ * Everything else in this library works out of a workspace that the caller allocates.  Some
+ * callers cannot allocate device memory at all: code running inside a region where the CUDA
+ * allocator must not be called (for example between other libraries' captured or timed sections),
+ * plug-ins that are handed device buffers by a host framework but have no allocator of their own,
+ * or processes whose memory budget is fixed before they start.  For them this call performs the
+ * same stable counting sort as zeda_route (drop the slots that chose a zero expert, count the
+ * surviving pairs per normal expert, exclusive offsets, permutation ordered by expert then token)
+ * on top-K indices the caller already has, and keeps its scratch in a fixed array inside the
+ * library instead of a workspace.
+ *   topk_idx        dev [T, top_k] int32 candidate ids; ids >= n_real are zero experts (input)
+ *   expert_counts   dev [n_real] int32          expert_offsets  dev [n_real + 1] int32
+ *   perm            dev [T * top_k] int32, first P entries written      n_pairs  dev [1] int32
+ * All pointers are required and belong to the CURRENT device.  Limits: T <= ZEDA_STATIC_MAX_TOKENS
+ * and T * top_k <= ZEDA_STATIC_MAX_SLOTS, n_real <= 512, top_k <= 16; larger sizes are rejected
+ * with ZEDA_ERR_UNSUPPORTED and nothing is launched.  T == 0 returns ZEDA_OK and touches nothing.
+ * The scratch array (about 0.4 MB) is part of the library image: every GPU that loads the library
+ * holds it until the process exits.  The call makes no cudaMalloc / cudaFree and uses no
+ * allocating library routine; it enqueues a small memset and three kernels on `stream`.
+ * The first call on each device looks up the array's device address (one cudaGetSymbolAddress,
+ * with that device current); make that first call before any stream capture begins.
+ * All calls on a device share the one array, which keeps the previous call's contents: the call
+ * clears the words that must start at zero itself, but two calls whose work overlaps on the GPU
+ * (different streams, or threads) race on it.  Serialise them on one stream. */
+#define ZEDA_STATIC_MAX_TOKENS 4096
+#define ZEDA_STATIC_MAX_SLOTS 32768
+zeda_status_t zeda_compact_static(const int32_t *topk_idx, int32_t T, int32_t top_k, int32_t n_real,
+                                  int32_t *expert_counts, int32_t *expert_offsets, int32_t *perm,
+                                  int32_t *n_pairs, void *stream);
+
 /* Reports a pending device-side error word (ZEDA_ERR_TIMEOUT) if any, then releases the handle.
  * Does not touch caller-owned device memory. */
 zeda_status_t zeda_moe_destroy(zeda_moe_t *h);

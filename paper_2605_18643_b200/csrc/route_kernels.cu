@@ -431,3 +431,81 @@ int launch_stats(const zeda_moe *h, const float *logits, const int32_t *topk_idx
 }
 
 }  // namespace zeda
+
+// ---------------------------------------------------------------------------------------------
+// zeda_compact_static: the counting sort above for callers that cannot allocate device memory.
+// Its scratch (per-CTA histograms, slot -> position table, pair -> token table, work lists,
+// counters) lives in the fixed array below instead of a caller-provided workspace.  Every GPU
+// that loads this library holds the array until the process exits.
+// ---------------------------------------------------------------------------------------------
+namespace zeda {
+namespace {
+
+constexpr int kStaticMaxTokens = ZEDA_STATIC_MAX_TOKENS;
+constexpr int kStaticMaxSlots = ZEDA_STATIC_MAX_SLOTS;
+constexpr int kStaticBlocks = (kStaticMaxTokens + kSortTokens - 1) / kSortTokens;
+constexpr int kStaticLists = kStaticMaxSlots / kChunkRows + kMaxCand + 1;
+
+struct StaticScratch {
+    int32_t block_hist[kStaticBlocks * kMaxCand];
+    int32_t inv[kStaticMaxSlots];
+    int32_t pair_token[kStaticMaxSlots];
+    int32_t chunk_expert[kStaticLists];
+    int32_t chunk_row0[kStaticLists];
+    int32_t tile_expert[kStaticLists];
+    int32_t tile_row0[kStaticLists];
+    int32_t meta[kMetaCount];
+};
+
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+constexpr int kMaxDevices = 64;
+StaticScratch *g_static_ptr[kMaxDevices] = {};  // device address of the array, per device
+
+}  // namespace
+}  // namespace zeda
+
+extern "C" zeda_status_t zeda_compact_static(const int32_t *topk_idx, int32_t T, int32_t top_k, int32_t n_real,
+                                             int32_t *expert_counts, int32_t *expert_offsets, int32_t *perm,
+                                             int32_t *n_pairs, void *stream) {
+    using namespace zeda;
+    if (T == 0) return ZEDA_OK;
+    if (T < 0 || T > kStaticMaxTokens || top_k < 1 || top_k > kMaxTopK || (long long)T * top_k > kStaticMaxSlots) {
+        set_error("zeda_compact_static handles at most %d tokens and %d slots (T * top_k); got T=%d, top_k=%d",
+                  kStaticMaxTokens, kStaticMaxSlots, T, top_k);
+        return ZEDA_ERR_UNSUPPORTED;
+    }
+    if (n_real < 1 || n_real > kMaxCand) { set_error("n_real must be in [1, %d]", kMaxCand); return ZEDA_ERR_UNSUPPORTED; }
+    if (!topk_idx || !expert_counts || !expert_offsets || !perm || !n_pairs) {
+        set_error("zeda_compact_static: every pointer is required");
+        return ZEDA_ERR_INVALID_ARG;
+    }
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { set_error("cudaGetDevice: %s", cudaGetErrorString(e)); return ZEDA_ERR_CUDA; }
+    if (dev < 0 || dev >= kMaxDevices) { set_error("device ordinal %d not supported", dev); return ZEDA_ERR_UNSUPPORTED; }
+    if (!g_static_ptr[dev]) {
+        // One-time set-up for this device: in host code the array's name is only a stand-in, the
+        // kernels need its device address.
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess || !p) { set_error("cudaGetSymbolAddress: %s", cudaGetErrorString(e)); return ZEDA_ERR_CUDA; }
+        g_static_ptr[dev] = static_cast<StaticScratch *>(p);
+    }
+    StaticScratch *sc = g_static_ptr[dev];
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the array keeps the previous call's contents; the counters start from zero every call
+    e = cudaMemsetAsync(sc->meta, 0, sizeof(sc->meta), s);
+    if (e != cudaSuccess) { set_error("cudaMemsetAsync: %s", cudaGetErrorString(e)); return ZEDA_ERR_CUDA; }
+    const int nblk = (T + kSortTokens - 1) / kSortTokens;
+    slot_hist_kernel<<<nblk, 256, sizeof(int32_t) * n_real, s>>>(topk_idx, T, top_k, n_real, sc->block_hist);
+    expert_scan_kernel<<<1, 512, 0, s>>>(sc->block_hist, nblk, n_real, T * top_k, expert_counts, expert_offsets,
+                                         n_pairs, sc->meta, sc->chunk_expert, sc->chunk_row0, sc->tile_expert,
+                                         sc->tile_row0);
+    slot_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * kPlaceWarps * n_real, s>>>(
+        topk_idx, T, top_k, n_real, sc->block_hist, expert_offsets, perm, nullptr, sc->inv, sc->pair_token);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { set_error("zeda_compact_static launch: %s", cudaGetErrorString(e)); return ZEDA_ERR_CUDA; }
+    return ZEDA_OK;
+}
+

@@ -24,7 +24,7 @@ FLAG_NONE, FLAG_FORCE_STREAM_EXPERTS, FLAG_FORCE_TILE_EXPERTS = 0, 1, 2
 EXPORTS = (
     "zeda_moe_workspace_bytes", "zeda_moe_create", "zeda_route", "zeda_route_from_logits",
     "zeda_router_logits", "zeda_moe_forward", "zeda_moe_forward_host", "zeda_moe_stats",
-    "zeda_moe_last_counters", "zeda_moe_set_profiling", "zeda_moe_stage_ms", "zeda_moe_destroy", "zeda_last_error", "zeda_version",
+    "zeda_moe_last_counters", "zeda_moe_set_profiling", "zeda_moe_stage_ms", "zeda_compact_static", "zeda_moe_destroy", "zeda_last_error", "zeda_version",
 )
 
 
@@ -69,6 +69,8 @@ def _load() -> ctypes.CDLL:
     lib.zeda_moe_set_profiling.argtypes = [vp, i32]
     lib.zeda_moe_stage_ms.restype = i32
     lib.zeda_moe_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    lib.zeda_compact_static.restype = i32
+    lib.zeda_compact_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.zeda_moe_destroy.restype = i32
     lib.zeda_moe_destroy.argtypes = [vp]
     lib.zeda_last_error.restype = ctypes.c_char_p
@@ -102,6 +104,26 @@ def _stream(device) -> ctypes.c_void_p:
 
 def workspace_bytes(cfg: Config) -> int:
     return int(lib.zeda_moe_workspace_bytes(ctypes.byref(cfg)))
+
+
+STATIC_MAX_TOKENS, STATIC_MAX_SLOTS = 4096, 32768
+
+
+def compact_static(topk_idx: torch.Tensor, n_real: int):
+    """zeda_compact_static: the counting sort of ``route`` for callers that cannot allocate device
+    memory; scratch lives in a fixed array inside the library.  The four output tensors made here
+    stand for buffers such a caller would already own.  Returns (counts, offsets, perm, n_pairs)."""
+    assert topk_idx.is_cuda and topk_idx.dtype == torch.int32 and topk_idx.is_contiguous() and topk_idx.dim() == 2
+    T, K = topk_idx.shape
+    dev = topk_idx.device
+    counts = torch.empty(n_real, dtype=torch.int32, device=dev)
+    offsets = torch.empty(n_real + 1, dtype=torch.int32, device=dev)
+    perm = torch.full((T * K,), -1, dtype=torch.int32, device=dev)
+    n_pairs = torch.zeros(1, dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        _check(lib.zeda_compact_static(_ptr(topk_idx), T, K, n_real, _ptr(counts), _ptr(offsets), _ptr(perm),
+                                       _ptr(n_pairs), _stream(dev)))
+    return counts, offsets, perm, n_pairs
 
 
 class ZedaMoE:
