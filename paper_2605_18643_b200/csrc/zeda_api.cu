@@ -74,6 +74,7 @@ size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int
     // pair buffers carry kTileM rows of slack so that a full tile may be stored past the last pair
     w.hmid = (__nv_bfloat16 *)take((slots + kTileM) * c.d_expert * 2);
     w.obuf = (__nv_bfloat16 *)take((slots + kTileM) * c.d_model * 2);
+    w.x_sorted = (__nv_bfloat16 *)take((slots + kTileM) * c.d_model * 2);
     w.x_stage = (__nv_bfloat16 *)take((size_t)c.max_tokens * c.d_model * 2);
     w.y_stage = (__nv_bfloat16 *)take((size_t)c.max_tokens * c.d_model * 2);
     if (ws) *ws = w;
@@ -126,11 +127,17 @@ zeda_status_t forward_device(zeda_moe_t *h, const __nv_bfloat16 *x, int T, __nv_
     if (r < 0) return cuda_fail("routing launch", cudaGetLastError());
     n += r;
     mark(2);
-    r = launch_experts_gemm1(h, x, T, s);
+    const bool tile = !(h->cfg.flags & ZEDA_FLAG_FORCE_STREAM_EXPERTS);
+    if (tile) {
+        r = launch_gather_rows(h, x, T, s);
+        if (r < 0) return cuda_fail("row gather launch", cudaGetLastError());
+        n += r;
+    }
+    r = tile ? launch_experts_gemm1_tile(h, T, s) : launch_experts_gemm1(h, x, T, s);
     if (r < 0) return cuda_fail("expert GEMM1 launch", cudaGetLastError());
     n += r;
     mark(3);
-    r = launch_experts_gemm2(h, T, s);
+    r = tile ? launch_experts_gemm2_tile(h, T, s) : launch_experts_gemm2(h, T, s);
     if (r < 0) return cuda_fail("expert GEMM2 launch", cudaGetLastError());
     n += r;
     mark(4);
@@ -200,6 +207,7 @@ zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_
     for (auto &ev : h->ev) ev = nullptr;
     carve(*cfg, static_cast<unsigned char *>(workspace), &h->ws, &h->max_chunks, &h->max_tiles);
     if (init_route_kernels(h) < 0) { delete h; return cuda_fail("kernel set-up", cudaGetLastError()); }
+    if (init_tile_kernels(h) < 0) { delete h; return ZEDA_ERR_CUDA; }
     e = cudaMemset(h->ws.meta, 0, kMetaCount * 4);
     if (e != cudaSuccess) { delete h; return cuda_fail("cudaMemset(meta)", e); }
     e = cudaDeviceSynchronize();

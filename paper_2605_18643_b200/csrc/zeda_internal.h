@@ -45,6 +45,7 @@ struct Workspace {
     float *stat_part;      // [nblk_stats * 2 * (N+N_Z)]
     __nv_bfloat16 *hmid;   // [maxT*K, He]
     __nv_bfloat16 *obuf;   // [maxT*K, d]
+    __nv_bfloat16 *x_sorted; // [maxT*K, d] x rows in pair order (tile path)
     __nv_bfloat16 *x_stage;// [maxT, d]
     __nv_bfloat16 *y_stage;// [maxT, d]
 };
@@ -87,6 +88,10 @@ int launch_stats(const zeda_moe *h, const float *logits, const int32_t *topk_idx
                  float *p_mean, float *out, cudaStream_t s);
 int launch_experts_gemm1(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
 int launch_experts_gemm2(const zeda_moe *h, int T, cudaStream_t s);
+int init_tile_kernels(zeda_moe *h);
+int launch_gather_rows(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
+int launch_experts_gemm1_tile(const zeda_moe *h, int T, cudaStream_t s);
+int launch_experts_gemm2_tile(const zeda_moe *h, int T, cudaStream_t s);
 int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s);
 
 void set_error(const char *fmt, ...);
