@@ -33,7 +33,7 @@ def _stale(target, deps):
 def build_library(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "nvcc")
     os.makedirs(OBJ, exist_ok=True)
-    headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".h")] + \
+    headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))] + \
               [os.path.join(ROOT, "include", "zeda.h"), os.path.abspath(__file__)]
     jobs = []
     objs = []

@@ -37,10 +37,11 @@ combine_kernel(const __nv_bfloat16 *__restrict__ obuf, const int32_t *__restrict
         s_zero_mass = zm;
     }
     __syncthreads();
-    for (int c = threadIdx.x; c < d / 8; c += blockDim.x) {
+    for (int c = blockIdx.y * blockDim.x + threadIdx.x; c < d / 8; c += gridDim.y * blockDim.x) {
         float acc[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+#pragma unroll 4
         for (int k = 0; k < K; ++k) {
             const int p = s_pos[k];
             if (p >= 0) fma_bf16x8(acc, s_w[k], __ldg(reinterpret_cast<const uint4 *>(obuf + (size_t)p * d) + c));
@@ -62,8 +63,11 @@ combine_kernel(const __nv_bfloat16 *__restrict__ obuf, const int32_t *__restrict
 
 int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s) {
     const zeda_moe_config_t &c = h->cfg;
-    const int threads = c.d_model / 8 >= 256 ? 256 : (c.d_model / 8 >= 128 ? 128 : 64);
-    combine_kernel<<<T, threads, 0, s>>>(h->ws.obuf, h->ws.inv, h->ws.topk_w, x, c.top_k, c.d_model,
+    // one 16-byte chunk per thread; small batches spread a row over several CTAs to fill the SMs
+    const int chunks = c.d_model / 8;
+    const int threads = (T >= 1024 && chunks >= 256) ? 256 : (T >= 256 && chunks >= 128 ? 128 : 64);
+    const int gy = (chunks + threads - 1) / threads;
+    combine_kernel<<<dim3(T, gy), threads, 0, s>>>(h->ws.obuf, h->ws.inv, h->ws.topk_w, x, c.top_k, c.d_model,
                                          c.expert_kind == ZEDA_EXPERT_COPY, y);
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }

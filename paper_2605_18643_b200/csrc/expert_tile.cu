@@ -17,13 +17,13 @@
 // Warp 0: TMA producer.  Warp 1: TMEM allocation + MMA issue.  Warps 2-5: epilogue (TMEM ->
 // registers -> SwiGLU / store).  Every mbarrier wait is bounded; on expiry the CTA records an
 // error word, lets its copies land, frees its TMEM and returns.
-#include <cuda.h>
-
-#include "zeda_internal.h"
+#include "tc_common.cuh"
 
 namespace zeda {
 
 namespace {
+
+using namespace tc;
 
 constexpr int kBlockK = 64;                  // bf16 elements per k-step = one 128-byte swizzle row
 constexpr int kATileBytes = 128 * kBlockK * 2;  // 16 KB
@@ -32,7 +32,6 @@ constexpr int kBBoxBytes = kBBoxRows * kBlockK * 2;  // 2 KB
 constexpr int kAccCols = 128;                // TMEM columns per accumulator
 constexpr int kTmemCols = 512;               // 2 buffers x 2 accumulators x 128 columns
 constexpr int kThreads = 192;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 struct TileMaps {
     CUtensorMap w_gate_up;  // [N][2He][d]  box {64, 128, 1}
@@ -40,123 +39,6 @@ struct TileMaps {
     CUtensorMap x_sorted;   // [rows][d]    box {64, 16}
     CUtensorMap hmid;       // [rows][He]   box {64, 16}
 };
-
-// ------------------------------------------------------------------------------------- PTX
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-
-// Bounded wait: false if the limit passed or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    if (mbar_try(bar, parity)) return true;
-    const unsigned long long t0 = globaltimer_ns();
-    int spins = 0;
-    while (!mbar_try(bar, parity)) {
-        if ((++spins & 63) == 0) {
-            if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > kWaitLimitNs) return false;
-        }
-    }
-    return true;
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, M = 128, N from the descriptor.
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-// mbarrier arrive once every MMA issued so far by this thread has finished (reads of smem done).
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-// 32 lanes x 32 columns of fp32 from TMEM: register j of lane i = D[lane_base + i][col + j].
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-    uint32_t r[32];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-}
-
-// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64 elements)
-// with the 128-byte swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3fffu);   // start address, 16-byte units
-    d |= (uint64_t)1 << 16;                   // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;         // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                   // descriptor version (sm_100)
-    d |= (uint64_t)2 << 61;                   // 128-byte swizzle
-    return d;
-}
-
-// kind::f16 instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128.
-__device__ __forceinline__ uint32_t instr_desc(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-}
 
 __device__ __forceinline__ float silu(float a) { return a / (1.f + expf(-a)); }
 
@@ -360,34 +242,6 @@ gather_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__restric
     }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-bool encode_bf16(CUtensorMap *m, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides_bytes,
-                 const cuuint32_t *box) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) { set_error("cuTensorMapEncodeTiled is not available from the driver"); return false; }
-    cuuint32_t ones[3] = {1, 1, 1};
-    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), dims, strides_bytes,
-                    box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed with code %d", (int)r); return false; }
-    return true;
-}
-
 template <int MODE, int TN_MAX, int STAGES>
 constexpr int tile_smem_bytes() { return STAGES * (2 * kATileBytes + TN_MAX * kBlockK * 2) + 1024; }
 
@@ -412,25 +266,25 @@ int init_tile_kernels(zeda_moe *h) {
         const cuuint64_t dims[3] = {d, 2 * He, E};
         const cuuint64_t strides[2] = {d * 2, 2 * He * d * 2};
         const cuuint32_t box[3] = {kBlockK, 128, 1};
-        ok = ok && encode_bf16(&tm->w_gate_up, h->w_gate_up, 3, dims, strides, box);
+        ok = ok && encode_bf16_map(&tm->w_gate_up, h->w_gate_up, 3, dims, strides, box);
     }
     {
         const cuuint64_t dims[3] = {He, d, E};
         const cuuint64_t strides[2] = {He * 2, d * He * 2};
         const cuuint32_t box[3] = {kBlockK, 128, 1};
-        ok = ok && encode_bf16(&tm->w_down, h->w_down, 3, dims, strides, box);
+        ok = ok && encode_bf16_map(&tm->w_down, h->w_down, 3, dims, strides, box);
     }
     {
         const cuuint64_t dims[2] = {d, rows};
         const cuuint64_t strides[1] = {d * 2};
         const cuuint32_t box[2] = {kBlockK, kBBoxRows};
-        ok = ok && encode_bf16(&tm->x_sorted, h->ws.x_sorted, 2, dims, strides, box);
+        ok = ok && encode_bf16_map(&tm->x_sorted, h->ws.x_sorted, 2, dims, strides, box);
     }
     {
         const cuuint64_t dims[2] = {He, rows};
         const cuuint64_t strides[1] = {He * 2};
         const cuuint32_t box[2] = {kBlockK, kBBoxRows};
-        ok = ok && encode_bf16(&tm->hmid, h->ws.hmid, 2, dims, strides, box);
+        ok = ok && encode_bf16_map(&tm->hmid, h->ws.hmid, 2, dims, strides, box);
     }
     ok = ok && set_smem_attr<1, kSmallTN, kSmallStages>() && set_smem_attr<2, kSmallTN, kSmallStages>() &&
          set_smem_attr<1, kBigTN, kBigStages>() && set_smem_attr<2, kBigTN, kBigStages>();

@@ -1,6 +1,8 @@
 // Routing stage: router logits over the N + N_Z candidates, softmax / top-K / routing weights
 // (Section 2.1), then the compaction that drops zero-expert slots and counting-sorts the surviving
 // (token, normal expert) pairs by expert in a stable order.
+#include <cooperative_groups.h>
+
 #include "zeda_internal.h"
 
 namespace zeda {
@@ -46,17 +48,25 @@ router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restric
 #pragma unroll
         for (int r = 0; r < kTok; ++r) acc[r] = 0.f;
         const float4 *wrow = reinterpret_cast<const float4 *>(router_w + (size_t)j * d);
-        for (int c4 = lane; c4 < d / 4; c4 += 32) {
-            const float4 w = __ldg(wrow + c4);
+        for (int c4 = lane; c4 < d / 4; c4 += 128) {
+            float4 w[4];
 #pragma unroll
-            for (int r = 0; r < kTok; ++r) {
-                const uint2 xv = reinterpret_cast<const uint2 *>(xs + (size_t)r * d)[c4];
-                const float x0 = __uint_as_float(xv.x << 16), x1 = __uint_as_float(xv.x & 0xffff0000u);
-                const float x2 = __uint_as_float(xv.y << 16), x3 = __uint_as_float(xv.y & 0xffff0000u);
-                acc[r] = fmaf(w.x, x0, acc[r]);
-                acc[r] = fmaf(w.y, x1, acc[r]);
-                acc[r] = fmaf(w.z, x2, acc[r]);
-                acc[r] = fmaf(w.w, x3, acc[r]);
+            for (int u = 0; u < 4; ++u)  // four independent 16-byte loads in flight per lane
+                w[u] = (c4 + 32 * u < d / 4) ? __ldg(wrow + c4 + 32 * u) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (c4 + 32 * u < d / 4) {
+#pragma unroll
+                    for (int r = 0; r < kTok; ++r) {
+                        const uint2 xv = reinterpret_cast<const uint2 *>(xs + (size_t)r * d)[c4 + 32 * u];
+                        const float x0 = __uint_as_float(xv.x << 16), x1 = __uint_as_float(xv.x & 0xffff0000u);
+                        const float x2 = __uint_as_float(xv.y << 16), x3 = __uint_as_float(xv.y & 0xffff0000u);
+                        acc[r] = fmaf(w[u].x, x0, acc[r]);
+                        acc[r] = fmaf(w[u].y, x1, acc[r]);
+                        acc[r] = fmaf(w[u].z, x2, acc[r]);
+                        acc[r] = fmaf(w[u].w, x3, acc[r]);
+                    }
+                }
             }
         }
         const float b = router_bias ? __ldg(router_bias + j) : 0.f;
@@ -75,42 +85,40 @@ router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restric
 // ---------------------------------------------------------------------------------------------
 constexpr int kRegsPerLane = kMaxCand / 32;
 
-__global__ void __launch_bounds__(256)
-topk_gate_kernel(const float *__restrict__ logits, int T, int n_real, int n_cand, int K, int gate_mode,
-                 int32_t *__restrict__ topk_idx, float *__restrict__ topk_w) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int t = blockIdx.x * (blockDim.x >> 5) + warp;
-    if (t >= T) return;
-    float v[kRegsPerLane];
-    const float *row = logits + (size_t)t * n_cand;
+// Top-K and routing weights of one token by one warp.  On return lane k < K holds slot k.
+// RPL = logits per lane (32 * RPL >= n_cand).
+template <int RPL>
+__device__ __forceinline__ void topk_gate_token(const float *__restrict__ row, int n_real, int n_cand, int K,
+                                                int gate_mode, int lane, int &my_idx, float &my_w) {
+    float v[RPL];
 #pragma unroll
-    for (int r = 0; r < kRegsPerLane; ++r) {
+    for (int r = 0; r < RPL; ++r) {
         const int j = r * 32 + lane;
         v[r] = (j < n_cand) ? row[j] : -INFINITY;
     }
     // row maximum and softmax denominator over all candidates
     float m = v[0];
 #pragma unroll
-    for (int r = 1; r < kRegsPerLane; ++r) m = fmaxf(m, v[r]);
+    for (int r = 1; r < RPL; ++r) m = fmaxf(m, v[r]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, o));
     float den = 0.f;
 #pragma unroll
-    for (int r = 0; r < kRegsPerLane; ++r) {
+    for (int r = 0; r < RPL; ++r) {
         const int j = r * 32 + lane;
         if (j < n_cand) den += expf(v[r] - m);
     }
     den = warp_sum(den);
 
     unsigned taken = 0;  // bit r set: this lane's register r was already selected
-    int my_idx = -1;     // lane k keeps slot k
     float my_p = 0.f;
     float sum_sel = 0.f, sum_real = 0.f;
+    my_idx = -1;
     for (int k = 0; k < K; ++k) {
         float bv = -INFINITY;
         int bj = 0x7fffffff;
 #pragma unroll
-        for (int r = 0; r < kRegsPerLane; ++r) {
+        for (int r = 0; r < RPL; ++r) {
             const int j = r * 32 + lane;
             if (j < n_cand && !((taken >> r) & 1u) && (v[r] > bv || bj == 0x7fffffff)) { bv = v[r]; bj = j; }
         }
@@ -126,12 +134,24 @@ topk_gate_kernel(const float *__restrict__ logits, int T, int n_real, int n_cand
         if (bj < n_real) sum_real += p;
         if (lane == k) { my_idx = bj; my_p = p; }
     }
+    my_w = my_p;
+    if (gate_mode == ZEDA_GATE_TOPK_NORM) my_w = my_p / sum_sel;
+    else if (gate_mode == ZEDA_GATE_RENORM_REAL) my_w = (my_idx < n_real && sum_real > 0.f) ? my_p / sum_real : 0.f;
+}
+
+template <int RPL>
+__global__ void __launch_bounds__(256)
+topk_gate_kernel(const float *__restrict__ logits, int T, int n_real, int n_cand, int K, int gate_mode,
+                 int32_t *__restrict__ topk_idx, float *__restrict__ topk_w) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (t >= T) return;
+    int my_idx;
+    float my_w;
+    topk_gate_token<RPL>(logits + (size_t)t * n_cand, n_real, n_cand, K, gate_mode, lane, my_idx, my_w);
     if (lane < K) {
-        float w = my_p;
-        if (gate_mode == ZEDA_GATE_TOPK_NORM) w = my_p / sum_sel;
-        else if (gate_mode == ZEDA_GATE_RENORM_REAL) w = (my_idx < n_real && sum_real > 0.f) ? my_p / sum_real : 0.f;
         topk_idx[(size_t)t * K + lane] = my_idx;
-        topk_w[(size_t)t * K + lane] = w;
+        topk_w[(size_t)t * K + lane] = my_w;
     }
 }
 
@@ -158,33 +178,27 @@ slot_hist_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real,
 // Counting sort, pass 2 (one CTA): column-wise exclusive scan over the CTA histograms, expert
 // counts, exclusive offsets, P, U, and the work lists of the expert kernels.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(512)
-expert_scan_kernel(int32_t *__restrict__ block_hist, int nblk, int n_real, int total_slots,
-                   int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
-                   int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
-                   int32_t *__restrict__ chunk_expert, int32_t *__restrict__ chunk_row0,
-                   int32_t *__restrict__ tile_expert, int32_t *__restrict__ tile_row0) {
-    __shared__ int32_t s_cnt[kMaxCand];
-    __shared__ int32_t s_off[kMaxCand + 1];
-    __shared__ int32_t s_chunk[kMaxCand + 1];
-    __shared__ int32_t s_tile[kMaxCand + 1];
+struct ScanShared {
+    int32_t cnt[kMaxCand];
+    int32_t off[kMaxCand + 1];
+    int32_t chunk[kMaxCand + 1];
+    int32_t tile[kMaxCand + 1];
+};
+
+// From per-expert pair counts in sh.cnt: exclusive offsets, P, U, and the work lists of the expert
+// kernels.  Called by every thread of the CTA (blockDim.x >= n_real); contains CTA barriers.
+__device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, int total_slots,
+                                                   int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
+                                                   int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
+                                                   int32_t *__restrict__ chunk_expert, int32_t *__restrict__ chunk_row0,
+                                                   int32_t *__restrict__ tile_expert, int32_t *__restrict__ tile_row0) {
     const int e = threadIdx.x;
-    if (e < n_real) {
-        int run = 0;
-        for (int b = 0; b < nblk; ++b) {
-            const int c = block_hist[(size_t)b * n_real + e];
-            block_hist[(size_t)b * n_real + e] = run;  // pairs of expert e in earlier CTAs
-            run += c;
-        }
-        s_cnt[e] = run;
-    }
-    __syncthreads();
     if (threadIdx.x < 32) {
-        // warp 0 scans the three per-expert sequences in chunks of 32
+        // warp 0 scans the three per-expert sequences in steps of 32 with shuffle prefix sums
         int base_off = 0, base_chunk = 0, base_tile = 0, active = 0, max_rows = 0;
         for (int e0 = 0; e0 < n_real; e0 += 32) {
             const int i = e0 + threadIdx.x;
-            const int c = (i < n_real) ? s_cnt[i] : 0;
+            const int c = (i < n_real) ? sh.cnt[i] : 0;
             const int ch = (c + kChunkRows - 1) / kChunkRows;
             const int tl = (c + kTileM - 1) / kTileM;
             int so = c, sc = ch, st = tl;
@@ -196,9 +210,9 @@ expert_scan_kernel(int32_t *__restrict__ block_hist, int nblk, int n_real, int t
                 if ((int)threadIdx.x >= o) { so += a; sc += b; st += g; }
             }
             if (i < n_real) {
-                s_off[i] = base_off + so - c;
-                s_chunk[i] = base_chunk + sc - ch;
-                s_tile[i] = base_tile + st - tl;
+                sh.off[i] = base_off + so - c;
+                sh.chunk[i] = base_chunk + sc - ch;
+                sh.tile[i] = base_tile + st - tl;
             }
             base_off += __shfl_sync(kFull, so, 31);
             base_chunk += __shfl_sync(kFull, sc, 31);
@@ -210,9 +224,7 @@ expert_scan_kernel(int32_t *__restrict__ block_hist, int nblk, int n_real, int t
             max_rows = max(max_rows, mx);
         }
         if (threadIdx.x == 0) {
-            s_off[n_real] = base_off;
-            s_chunk[n_real] = base_chunk;
-            s_tile[n_real] = base_tile;
+            sh.off[n_real] = base_off;
             meta[kMetaPairs] = base_off;
             meta[kMetaActive] = active;
             meta[kMetaZeroSlots] = total_slots - base_off;
@@ -224,15 +236,105 @@ expert_scan_kernel(int32_t *__restrict__ block_hist, int nblk, int n_real, int t
     }
     __syncthreads();
     if (e < n_real) {
-        const int c = s_cnt[e];
+        const int c = sh.cnt[e];
         if (counts) counts[e] = c;
-        offsets[e] = s_off[e];
-        int ci = s_chunk[e];
+        offsets[e] = sh.off[e];
+        int ci = sh.chunk[e];
         for (int r = 0; r < c; r += kChunkRows, ++ci) { chunk_expert[ci] = e; chunk_row0[ci] = r; }
-        int ti = s_tile[e];
+        int ti = sh.tile[e];
         for (int r = 0; r < c; r += kTileM, ++ti) { tile_expert[ti] = e; tile_row0[ti] = r; }
     }
-    if (e == 0) offsets[n_real] = s_off[n_real];
+    if (e == 0) offsets[n_real] = sh.off[n_real];
+}
+
+__global__ void __launch_bounds__(512)
+expert_scan_kernel(int32_t *__restrict__ block_hist, int nblk, int n_real, int total_slots,
+                   int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
+                   int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
+                   int32_t *__restrict__ chunk_expert, int32_t *__restrict__ chunk_row0,
+                   int32_t *__restrict__ tile_expert, int32_t *__restrict__ tile_row0) {
+    __shared__ ScanShared sh;
+    const int e = threadIdx.x;
+    if (e < n_real) {
+        int run = 0;
+        for (int b = 0; b < nblk; ++b) {
+            const int c = block_hist[(size_t)b * n_real + e];
+            block_hist[(size_t)b * n_real + e] = run;  // pairs of expert e in earlier CTAs
+            run += c;
+        }
+        sh.cnt[e] = run;
+    }
+    __syncthreads();
+    finish_expert_scan(sh, n_real, total_slots, counts, offsets, n_pairs_out, meta, chunk_expert, chunk_row0,
+                       tile_expert, tile_row0);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Small batches (T <= 128, decode): top-K, routing weights and the whole counting sort in ONE
+// launch of a thread-block cluster.  Each CTA of the cluster takes 16 tokens (one warp per token)
+// and records "token t selected expert e" as bit t of a T-bit mask that lives in CTA 0's shared
+// memory (distributed shared memory, atomicOr).  A token selects an expert at most once, so an
+// expert's count is a popcount and the stable rank of a pair is the popcount of the lower token
+// bits: the (expert, token) order needs no atomics on positions and no second pass.  After the
+// cluster barrier CTA 0 scans the experts and places the pairs.
+// ---------------------------------------------------------------------------------------------
+constexpr int kSmallTokens = 128;
+constexpr int kSmallCluster = 8;
+constexpr int kSmallThreads = 32 * (kSmallTokens / kSmallCluster);  // one warp per token
+
+template <int RPL>
+__global__ void __cluster_dims__(kSmallCluster, 1, 1) __launch_bounds__(kSmallThreads)
+route_small_kernel(const float *__restrict__ logits, int T, int n_real, int n_cand, int K, int gate_mode,
+                   int32_t *__restrict__ topk_idx, float *__restrict__ topk_w, int32_t *__restrict__ counts,
+                   int32_t *__restrict__ offsets, int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
+                   int32_t *__restrict__ chunk_expert, int32_t *__restrict__ chunk_row0,
+                   int32_t *__restrict__ tile_expert, int32_t *__restrict__ tile_row0, int32_t *__restrict__ perm,
+                   int32_t *__restrict__ perm_user, int32_t *__restrict__ inv, int32_t *__restrict__ pair_token) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    __shared__ ScanShared sh;
+    __shared__ uint32_t sel[kMaxCand][kSmallTokens / 32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned rank = cluster.block_rank();
+    if (rank == 0)
+        for (int i = threadIdx.x; i < n_real * (kSmallTokens / 32); i += blockDim.x) (&sel[0][0])[i] = 0u;
+    cluster.sync();
+    uint32_t *sel0 = cluster.map_shared_rank(&sel[0][0], 0);
+    const int t = rank * (kSmallThreads / 32) + warp;
+    if (t < T) {
+        int my_idx;
+        float my_w;
+        topk_gate_token<RPL>(logits + (size_t)t * n_cand, n_real, n_cand, K, gate_mode, lane, my_idx, my_w);
+        if (lane < K) {
+            topk_idx[(size_t)t * K + lane] = my_idx;
+            topk_w[(size_t)t * K + lane] = my_w;
+            if (my_idx < n_real) atomicOr(sel0 + my_idx * (kSmallTokens / 32) + (t >> 5), 1u << (t & 31));
+        }
+    }
+    cluster.sync();  // release/acquire at cluster scope: masks and topk_idx of every CTA are visible
+    if (rank != 0) return;
+    if ((int)threadIdx.x < n_real) {
+        int c = 0;
+#pragma unroll
+        for (int i = 0; i < kSmallTokens / 32; ++i) c += __popc(sel[threadIdx.x][i]);
+        sh.cnt[threadIdx.x] = c;
+    }
+    __syncthreads();
+    finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, chunk_expert, chunk_row0, tile_expert,
+                       tile_row0);
+    for (int s = threadIdx.x; s < T * K; s += blockDim.x) {
+        const int e = topk_idx[s], tk = s / K;
+        int p = -1;
+        if (e < n_real) {
+            int r = __popc(sel[e][tk >> 5] & ((1u << (tk & 31)) - 1u));
+            for (int i = 0; i < (tk >> 5); ++i) r += __popc(sel[e][i]);
+            p = sh.off[e] + r;
+            perm[p] = s;
+            if (perm_user) perm_user[p] = s;
+            pair_token[p] = tk;
+        }
+        inv[s] = p;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -384,6 +486,8 @@ int init_route_kernels(const zeda_moe *h) {
 }
 
 int launch_router_logits(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, cudaStream_t s) {
+    // large batches: the GEMM goes to the tensor cores (exact three-way bf16 split of the weights)
+    if (T >= 256 && h->router_maps) return launch_router_logits_tile(h, x, T, logits, s);
     const int d = h->cfg.d_model, n_cand = h->cfg.n_real + h->cfg.n_zero;
     const int tiles = (T + kTok - 1) / kTok;
     // split the candidates over grid.y until the grid covers the SMs about twice
@@ -403,12 +507,34 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
     const int n_cand = c.n_real + c.n_zero, K = c.top_k;
     const Workspace &ws = h->ws;
     const int nblk = (T + kSortTokens - 1) / kSortTokens;
-    topk_gate_kernel<<<(T + 7) / 8, 256, 0, s>>>(logits, T, c.n_real, n_cand, K, c.gate_mode, ws.topk_idx, ws.topk_w);
-    slot_hist_kernel<<<nblk, 256, sizeof(int32_t) * c.n_real, s>>>(ws.topk_idx, T, K, c.n_real, ws.block_hist);
-    expert_scan_kernel<<<1, 512, 0, s>>>(ws.block_hist, nblk, c.n_real, T * K, ws.counts, ws.offsets, out.n_pairs,
-                                         ws.meta, ws.chunk_expert, ws.chunk_row0, ws.tile_expert, ws.tile_row0);
-    slot_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * kPlaceWarps * c.n_real, s>>>(
-        ws.topk_idx, T, K, c.n_real, ws.block_hist, ws.offsets, ws.perm, out.perm, ws.inv, ws.pair_token);
+    int launches = 4;
+#define ZEDA_RPL_DISPATCH(CALL)                        \
+    do {                                               \
+        if (n_cand <= 64) { CALL(2); }                 \
+        else if (n_cand <= 128) { CALL(4); }           \
+        else if (n_cand <= 256) { CALL(8); }           \
+        else { CALL(16); }                             \
+    } while (0)
+    if (T <= kSmallTokens && c.n_real <= kSmallThreads) {
+#define ZEDA_CALL_SMALL(R)                                                                                         \
+    route_small_kernel<R><<<kSmallCluster, kSmallThreads, 0, s>>>(                                                 \
+        logits, T, c.n_real, n_cand, K, c.gate_mode, ws.topk_idx, ws.topk_w, ws.counts, ws.offsets, out.n_pairs,   \
+        ws.meta, ws.chunk_expert, ws.chunk_row0, ws.tile_expert, ws.tile_row0, ws.perm, out.perm, ws.inv,          \
+        ws.pair_token)
+        ZEDA_RPL_DISPATCH(ZEDA_CALL_SMALL);
+#undef ZEDA_CALL_SMALL
+        launches = 1;
+    } else {
+#define ZEDA_CALL_TOPK(R) \
+    topk_gate_kernel<R><<<(T + 7) / 8, 256, 0, s>>>(logits, T, c.n_real, n_cand, K, c.gate_mode, ws.topk_idx, ws.topk_w)
+        ZEDA_RPL_DISPATCH(ZEDA_CALL_TOPK);
+#undef ZEDA_CALL_TOPK
+        slot_hist_kernel<<<nblk, 256, sizeof(int32_t) * c.n_real, s>>>(ws.topk_idx, T, K, c.n_real, ws.block_hist);
+        expert_scan_kernel<<<1, 512, 0, s>>>(ws.block_hist, nblk, c.n_real, T * K, ws.counts, ws.offsets, out.n_pairs,
+                                             ws.meta, ws.chunk_expert, ws.chunk_row0, ws.tile_expert, ws.tile_row0);
+        slot_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * kPlaceWarps * c.n_real, s>>>(
+            ws.topk_idx, T, K, c.n_real, ws.block_hist, ws.offsets, ws.perm, out.perm, ws.inv, ws.pair_token);
+    }
     if (cudaGetLastError() != cudaSuccess) return -1;
     // copies for a caller that asked for the routing itself
     const cudaMemcpyKind d2d = cudaMemcpyDeviceToDevice;
@@ -416,7 +542,7 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
     if (out.topk_w) cudaMemcpyAsync(out.topk_w, ws.topk_w, sizeof(float) * (size_t)T * K, d2d, s);
     if (out.counts) cudaMemcpyAsync(out.counts, ws.counts, sizeof(int32_t) * c.n_real, d2d, s);
     if (out.offsets) cudaMemcpyAsync(out.offsets, ws.offsets, sizeof(int32_t) * (c.n_real + 1), d2d, s);
-    return cudaGetLastError() == cudaSuccess ? 4 : -1;
+    return cudaGetLastError() == cudaSuccess ? launches : -1;
 }
 
 int launch_stats(const zeda_moe *h, const float *logits, const int32_t *topk_idx, int T, float *f,

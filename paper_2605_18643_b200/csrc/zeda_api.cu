@@ -74,6 +74,7 @@ size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int
     // pair buffers carry kTileM rows of slack so that a full tile may be stored past the last pair
     w.hmid = (__nv_bfloat16 *)take((slots + kTileM) * c.d_expert * 2);
     w.obuf = (__nv_bfloat16 *)take((slots + kTileM) * c.d_model * 2);
+    w.router_split = (__nv_bfloat16 *)take((size_t)3 * router_split_pad((int)n_cand) * c.d_model * 2);
     w.x_sorted = (__nv_bfloat16 *)take((slots + kTileM) * c.d_model * 2);
     w.x_stage = (__nv_bfloat16 *)take((size_t)c.max_tokens * c.d_model * 2);
     w.y_stage = (__nv_bfloat16 *)take((size_t)c.max_tokens * c.d_model * 2);
@@ -202,12 +203,18 @@ zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_
     h->sm_count = prop.multiProcessorCount;
     h->last_launches = 0;
     h->tmaps = nullptr;
+    h->router_maps = nullptr;
     h->profiling = false;
     h->profiled_last = false;
     for (auto &ev : h->ev) ev = nullptr;
     carve(*cfg, static_cast<unsigned char *>(workspace), &h->ws, &h->max_chunks, &h->max_tiles);
     if (init_route_kernels(h) < 0) { delete h; return cuda_fail("kernel set-up", cudaGetLastError()); }
     if (init_tile_kernels(h) < 0) { delete h; return ZEDA_ERR_CUDA; }
+    if (init_router_tile(h) < 0) {
+        if (h->tmaps) free(h->tmaps);
+        delete h;
+        return cuda_fail("router set-up", cudaGetLastError());
+    }
     e = cudaMemset(h->ws.meta, 0, kMetaCount * 4);
     if (e != cudaSuccess) { delete h; return cuda_fail("cudaMemset(meta)", e); }
     e = cudaDeviceSynchronize();
@@ -351,6 +358,7 @@ zeda_status_t zeda_moe_destroy(zeda_moe_t *h) {
     }
     for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
     if (h->tmaps) free(h->tmaps);
+    if (h->router_maps) free(h->router_maps);
     delete h;
     return st;
 }

@@ -45,6 +45,7 @@ struct Workspace {
     float *stat_part;      // [nblk_stats * 2 * (N+N_Z)]
     __nv_bfloat16 *hmid;   // [maxT*K, He]
     __nv_bfloat16 *obuf;   // [maxT*K, d]
+    __nv_bfloat16 *router_split; // [3][pad128(N+N_Z)][d] bf16 hi/mid/lo pieces of the router rows
     __nv_bfloat16 *x_sorted; // [maxT*K, d] x rows in pair order (tile path)
     __nv_bfloat16 *x_stage;// [maxT, d]
     __nv_bfloat16 *y_stage;// [maxT, d]
@@ -73,6 +74,7 @@ struct zeda_moe {
     int max_tiles;
     int last_launches;
     void *tmaps;  // host-side tensor maps of the tile path (owned)
+    void *router_maps;  // host-side tensor map of the split router weights (owned)
     bool profiling;
     bool profiled_last;
     cudaEvent_t ev[ZEDA_STAGE_COUNT + 1];
@@ -89,6 +91,9 @@ int launch_stats(const zeda_moe *h, const float *logits, const int32_t *topk_idx
 int launch_experts_gemm1(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
 int launch_experts_gemm2(const zeda_moe *h, int T, cudaStream_t s);
 int init_tile_kernels(zeda_moe *h);
+int router_split_pad(int n_cand);
+int init_router_tile(zeda_moe *h);
+int launch_router_logits_tile(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, cudaStream_t s);
 int launch_gather_rows(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
 int launch_experts_gemm1_tile(const zeda_moe *h, int T, cudaStream_t s);
 int launch_experts_gemm2_tile(const zeda_moe *h, int T, cudaStream_t s);
