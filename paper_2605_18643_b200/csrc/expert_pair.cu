@@ -1,0 +1,475 @@
+// Grouped expert GEMMs on CTA pairs: tcgen05.mma.cta_group::2 (M = 256 over two SMs), accumulators
+// in TMEM, weights and Hmid staged in shared memory by TMA, the x rows of GEMM1 gathered straight
+// from the token-order x by cp.async (no gathered copy of x is ever written).
+//
+// Appendix D: each normal expert has gate, up and down projections; a surviving (token, expert)
+// pair costs 6*H*H_e FLOPs, a zero-expert slot none (it never reaches these kernels).  Both GEMMs
+// run "weights as the M operand": the 256 rows of the MMA are weight rows (128 in each CTA of the
+// pair), its N <= 256 columns are pair rows of ONE expert (N/2 loaded by each CTA), so a ragged
+// expert costs its pair count rounded up to 32 columns, and each CTA loads 128 weight rows plus at
+// most 128 activation rows per 128 x 256 block of outputs.
+//
+//   work item  = (expert e, block of <= 256 of its pair rows, block mb of weight rows)
+//   GEMM1      A tile of CTA r = 64 gate rows of 64-row block (2 mb + r) followed by the matching 64
+//              up rows (one 5-D TMA box); B = x rows of the pairs, fetched by four gather warps
+//              through pair_token with 16-byte cp.async into the 128-byte-swizzled layout; K = H.
+//              TMEM lanes 0-63 hold gate values, lanes 64-127 the up values of the same features;
+//              the epilogue warps swap halves through shared memory, apply SwiGLU and store Hmid.
+//   GEMM2      A tile of CTA r = 128 down rows [256 mb + 128 r, +128); B = Hmid rows; K = H_e.
+//
+// One CTA per SM, persistent over a device-side work list (the host never learns P or the counts).
+// Warp 0: TMA producer (weights).  Warp 1: TMEM allocation, and in the leader CTA the MMA issue.
+// Warp 2 (GEMM1): gather relay.  Warp 3 (GEMM2): TMA producer of the Hmid rows.  Warps 4-7:
+// epilogue.  Warps 8-11 (GEMM1): x-row gather.  Full barriers live in the leader CTA and count the
+// TMA bytes (and gather relays) of both CTAs; stage-empty and accumulator-full barriers are
+// signalled in both CTAs by multicast commits.  Every mbarrier wait is bounded; on expiry the CTA
+// records an error word, skips the rest of its work, and leaves through the common exit (cluster
+// barrier, TMEM free).
+#include "tc_common.cuh"
+
+namespace zeda {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kBlockK = 64;                     // bf16 elements per k-step = one 128-byte swizzle row
+constexpr int kATileBytes = 128 * kBlockK * 2;  // 16 KB: this CTA's 128 weight rows of one k-step
+constexpr int kRowBytes = kBlockK * 2;          // 128
+constexpr int kAccCols = 256;                   // TMEM columns of one accumulator buffer
+constexpr int kTmemCols = 512;                  // two buffers
+constexpr int kThreads = 256;                   // GEMM2
+constexpr int kThreadsGather = 384;             // GEMM1: + four gather warps
+constexpr int kPatchBytes = 4 * 32 * 32 * 2;    // per epilogue warp: [32 pair rows][32 features] bf16, for 16-byte stores
+constexpr int kXchgBytes = 2 * 2 * 32 * 32 * 4; // GEMM1 gate/up swap: [warp pair][direction][32 cols][32 lanes] fp32
+
+// Hmid row blocks come in boxes of 128, 64, 32 and 16 rows: a block of 16 k rows is loaded with
+// at most four TMA instructions (few large boxes: issuing a TMA instruction costs a few hundred cycles).
+struct RowMaps {
+    CUtensorMap m[4];  // box {64, 128 >> i}
+};
+
+struct PairMaps {
+    CUtensorMap w_gate_up;  // [N][He/64 blocks][gate | up][64 rows][d]  box {64, 64, 2, 1, 1}
+    CUtensorMap w_down;     // [N][d][He]   box {64, 128, 1}
+    RowMaps hmid;           // [rows][He]
+};
+
+struct Item {
+    int e, pos0, n, mb;
+};
+
+__device__ __forceinline__ Item load_item(long long item, int m_blocks, const int32_t *tile_expert,
+                                          const int32_t *tile_row0, const int32_t *counts, const int32_t *offsets) {
+    Item it;
+    const int tile = (int)(item / m_blocks);
+    it.mb = (int)(item % m_blocks);
+    it.e = tile_expert[tile];
+    const int r0 = tile_row0[tile];
+    it.n = min(kPairTileM, counts[it.e] - r0);
+    it.pos0 = offsets[it.e] + r0;
+    return it;
+}
+
+__device__ __forceinline__ void named_sync(int id, int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+__device__ __forceinline__ float swiglu(float g, float u) { return __fdividef(g * u, 1.f + __expf(-g)); }
+
+// MODE 1: GEMM1 + SwiGLU -> Hmid[pos, f].   MODE 2: GEMM2 -> O[pos, row].
+// HALF_MAX: most B rows one CTA loads per k-step (the tile's column count is at most 2 * HALF_MAX).
+template <int MODE, int HALF_MAX, int STAGES>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MODE == 1 ? kThreadsGather : kThreads, 1)
+expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ RowMaps maps_b,
+                        const __nv_bfloat16 *__restrict__ x, int x_ld, const int32_t *__restrict__ counts,
+                        const int32_t *__restrict__ offsets, const int32_t *__restrict__ tile_expert,
+                        const int32_t *__restrict__ tile_row0, const int32_t *__restrict__ pair_token,
+                        int32_t *__restrict__ meta, int kdim, int out_rows, int m_blocks,
+                        __nv_bfloat16 *__restrict__ out, int out_ld) {
+    constexpr int kStageBytes = kATileBytes + HALF_MAX * kRowBytes;
+    extern __shared__ __align__(1024) unsigned char pair_smem[];
+    __shared__ __align__(8) unsigned long long bars[3 * STAGES + 4];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+    __shared__ int s_ok[4];
+
+    // 1024-byte alignment of the operand ring (the swizzle pattern is a function of the address)
+    const uint32_t ring = (smem_u32(pair_smem) + 1023u) & ~1023u;
+    unsigned char *after_ring = pair_smem + (ring - smem_u32(pair_smem)) + STAGES * kStageBytes;
+    __nv_bfloat16 *patches = reinterpret_cast<__nv_bfloat16 *>(after_ring);
+    float *xchg = reinterpret_cast<float *>(after_ring + kPatchBytes);
+    const uint32_t bar_full = smem_u32(&bars[0]);                 // used in the leader CTA only
+    const uint32_t bar_empty = smem_u32(&bars[STAGES]);           // one set per CTA
+    const uint32_t bar_tfull = smem_u32(&bars[2 * STAGES]);       // one set per CTA
+    const uint32_t bar_tempty = smem_u32(&bars[2 * STAGES + 2]);  // used in the leader CTA only
+    const uint32_t bar_gfull = smem_u32(&bars[2 * STAGES + 4]);   // GEMM1: this CTA's gathered rows of a stage have landed
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        // full: the TMA producer's expect_tx arrival (+ GEMM1: the gather relay of each CTA)
+        for (int i = 0; i < STAGES; ++i) {
+            mbar_init(bar_full + 8 * i, MODE == 1 ? 3 : 1);
+            mbar_init(bar_empty + 8 * i, 1);
+            mbar_init(bar_gfull + 8 * i, 128);
+        }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar_tfull + 8 * i, 1); mbar_init(bar_tempty + 8 * i, 8); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc_pair(smem_u32(&s_tmem_base), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // both CTAs' barriers are initialised before any remote signal
+    tc_fence_after();
+    const uint32_t tmem_base = s_tmem_base;
+    volatile int *abort_flag = &s_abort;
+
+    const long long n_items = (long long)meta[kMetaPairTiles] * m_blocks;
+    const int k_steps = kdim / kBlockK;
+    const long long first = blockIdx.x >> 1, stride = gridDim.x >> 1;
+    const uint32_t full0 = mapa(bar_full, 0);      // the leader's full barriers, as seen from either CTA
+    const uint32_t tempty0 = mapa(bar_tempty, 0);  // the leader's accumulator-free barriers
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (weights)
+        if (lane == 0) {
+            uint32_t it_count = 0;
+            bool ok = true;
+            for (long long item = first; item < n_items && ok; item += stride) {
+                const Item it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
+                const int half = ((it.n + 31) >> 5) << 4;  // B rows of this CTA; the tile has 2 * half columns
+                const uint32_t bytes = 2u * (uint32_t)(kATileBytes + (MODE == 2 ? half * kRowBytes : 0));
+                for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
+                    const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
+                    if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t full = full0 + 8 * s;
+                    const uint32_t sa = ring + s * kStageBytes;
+                    if (leader) mbar_expect_tx(bar_full + 8 * s, bytes);  // the TMA bytes of both CTAs
+                    if (MODE == 1)  // one box: 64 gate rows of block (2 mb + rank), then the 64 up rows of the same block
+                        tma_load_5d_pair(sa, &map_a, ks * kBlockK, 0, 0, 2 * it.mb + (int)rank, it.e, full);
+                    else
+                        tma_load_3d_pair(sa, &map_a, ks * kBlockK, 256 * it.mb + 128 * (int)rank, it.e, full);
+                }
+            }
+            if (!ok) {
+                if (!*abort_flag) atomicExch(&meta[kMetaError], 11);
+                s_abort = 1;
+            }
+        }
+    } else if (MODE == 2 && warp == 3) {
+        // ------------------------------------------------------------------ TMA producer of the Hmid rows (GEMM2)
+        // A second issuing thread: one thread cannot issue the loads of both operands fast enough.
+        if (lane == 0) {
+            uint32_t it_count = 0;
+            bool ok = true;
+            for (long long item = first; item < n_items && ok; item += stride) {
+                const Item it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
+                const int half = ((it.n + 31) >> 5) << 4;
+                const int brow0 = (int)rank * half;  // first tile column / pair row this CTA loads
+                for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
+                    const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
+                    if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t full = full0 + 8 * s;
+                    const uint32_t sb = ring + s * kStageBytes + kATileBytes;
+                    int b = 0;
+#pragma unroll
+                    for (int lvl = 0; lvl < 4; ++lvl) {
+                        const int rows = 128 >> lvl;
+                        if (rows <= HALF_MAX && half - b >= rows) {
+                            tma_load_2d_pair(sb + b * kRowBytes, &maps_b.m[lvl], ks * kBlockK, it.pos0 + brow0 + b, full);
+                            b += rows;
+                        }
+                    }
+                }
+            }
+            if (!ok) {
+                if (!*abort_flag) atomicExch(&meta[kMetaError], 16);
+                s_abort = 1;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA)
+        if (leader && lane == 0) {
+            uint32_t it_count = 0, tile_count = 0;
+            bool ok = true;
+            for (long long item = first; item < n_items && ok; item += stride, ++tile_count) {
+                const Item it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
+                const int n_cols = ((it.n + 31) >> 5) << 5;
+                const uint32_t idesc = instr_desc_pair(n_cols);
+                const uint32_t buf = tile_count & 1u, tph = (tile_count >> 1) & 1u;
+                if (!mbar_wait(bar_tempty + 8 * buf, tph ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d = tmem_base + buf * kAccCols;
+                for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
+                    const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
+                    if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = ring + s * kStageBytes;
+                    const uint64_t a = smem_desc_sw128(sa);
+                    const uint64_t b = smem_desc_sw128(sa + kATileBytes);
+#pragma unroll
+                    for (int k = 0; k < kBlockK / 16; ++k)  // +32 bytes per 16-element k slice inside the swizzle row
+                        umma_bf16_pair(d, a + 2 * k, b + 2 * k, idesc, (ks | k) ? 1u : 0u);
+                    umma_commit_pair(bar_empty + 8 * s);  // the stage is free in both CTAs once these MMAs have read it
+                }
+                if (!ok) break;
+                umma_commit_pair(bar_tfull + 8 * buf);    // accumulators complete in both CTAs
+            }
+            if (!ok) {
+                if (!*abort_flag) atomicExch(&meta[kMetaError], 12);
+                s_abort = 1;
+            }
+        }
+    } else if (MODE == 1 && warp == 2) {
+        // ------------------------------------------------------------------ gather relay (GEMM1)
+        // cp.async can only signal an mbarrier of its own CTA: this thread forwards "this CTA's
+        // gathered rows of stage s have landed" to the leader's full barrier.
+        if (lane == 0) {
+            uint32_t it_count = 0;
+            bool ok = true;
+            for (long long item = first; item < n_items && ok; item += stride) {
+                for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
+                    const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
+                    if (!mbar_wait(bar_gfull + 8 * s, ph, abort_flag)) { ok = false; break; }
+                    mbar_arrive_cluster(full0 + 8 * s);
+                }
+            }
+            if (!ok) {
+                if (!*abort_flag) atomicExch(&meta[kMetaError], 15);
+                s_abort = 1;
+            }
+        }
+    } else if (MODE == 1 && warp >= 8) {
+        // ------------------------------------------------------------------ x-row gather (GEMM1)
+        // Thread gt copies 16-byte chunk (gt & 7) of rows (gt >> 3) + 16 i, i = 0..7, of this CTA's
+        // half of the tile's pair rows.  The chunk lands where the 128-byte swizzle puts it
+        // (chunk index XOR row mod 8).  Each thread's copies of a stage arrive on the stage's
+        // local barrier when they complete; nothing here waits for a copy.
+        const int gt = threadIdx.x - 256;
+        const int chunk = gt & 7, rsub = gt >> 3;
+        const uint32_t dst_off = (uint32_t)(rsub * kRowBytes + ((chunk ^ (rsub & 7)) << 4));
+        uint32_t it_count = 0;
+        bool ok = true;
+        for (long long item = first; item < n_items && ok; item += stride) {
+            const Item it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
+            const int half = ((it.n + 31) >> 5) << 4;
+            const int brow0 = (int)rank * half;
+            const __nv_bfloat16 *src[HALF_MAX / 16];
+#pragma unroll
+            for (int i = 0; i < HALF_MAX / 16; ++i) {
+                const int rb = brow0 + rsub + 16 * i;
+                // padding rows read token 0: their columns are never stored
+                const int tok = (rsub + 16 * i < half && rb < it.n) ? pair_token[it.pos0 + rb] : 0;
+                src[i] = x + (size_t)tok * x_ld + chunk * 8;
+            }
+            for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
+                const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
+                if (lane == 0) ok = mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag);
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                const uint32_t sb = ring + s * kStageBytes + kATileBytes + dst_off;
+#pragma unroll
+                for (int i = 0; i < HALF_MAX / 16; ++i)
+                    if (rsub + 16 * i < half) cp_async16(sb + i * 16 * kRowBytes, src[i] + ks * kBlockK);
+                cp_async_arrive_noinc(bar_gfull + 8 * s);
+            }
+        }
+        cp_async_wait_all();  // the copies issued so far land in this CTA before it may leave
+        if (!ok && lane == 0) {
+            if (!*abort_flag) atomicExch(&meta[kMetaError], 14);
+            s_abort = 1;
+        }
+    } else if (warp >= 4 && warp < 8) {
+        // ------------------------------------------------------------------ epilogue warps
+        const int q = warp & 3;      // TMEM lane quarter this warp may read
+        const int wp = q & 1;        // GEMM1: warp pair (gate warp q = wp, up warp q = wp + 2) sharing 32 features
+        const bool is_up = q >= 2;
+        __nv_bfloat16 *patch = patches + q * 1024;   // [32 pair rows][32 features]
+        const int prow = lane >> 2, pch = lane & 3;  // 16-byte piece this lane stores: rows prow + 8 i, features 8 pch ..
+        uint32_t tile_count = 0;
+        bool ok = true;
+        for (long long item = first; item < n_items && ok; item += stride, ++tile_count) {
+            const Item it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
+            const uint32_t buf = tile_count & 1u, tph = (tile_count >> 1) & 1u;
+            ok = mbar_wait(bar_tfull + 8 * buf, tph, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp before the aligned TMEM loads
+            if (MODE == 1) {
+                // the two warps of a pair meet at named barriers below: they must take the same branch
+                if (lane == 0) s_ok[q] = ok ? 1 : 0;
+                named_sync(1 + wp, 64);
+                ok = s_ok[wp] && s_ok[wp + 2];
+                named_sync(1 + wp, 64);
+            }
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t0 = tmem_base + ((uint32_t)(32 * q) << 16) + buf * kAccCols;
+            if (MODE == 1) {
+                const int f0 = 128 * it.mb + 64 * (int)rank + 32 * wp;  // first of this warp's 32 features
+                const bool f_ok = f0 < out_rows;
+                float *bw = xchg + (wp * 2 + (is_up ? 1 : 0)) * 1024;
+                const float *br = xchg + (wp * 2 + (is_up ? 0 : 1)) * 1024;
+                for (int c0 = 0; c0 < it.n; c0 += 64) {
+                    // the gate warp finishes columns [c0, c0+32), the up warp columns [c0+32, c0+64)
+                    uint32_t keep_u[32], send_u[32];
+                    tmem_ld32_nowait(t0 + c0 + (is_up ? 0 : 32), send_u);
+                    tmem_ld32_nowait(t0 + c0 + (is_up ? 32 : 0), keep_u);
+                    tmem_ld_wait();
+                    if (c0 + 64 >= it.n) {
+                        // last read of this buffer: hand it back to the MMA warp before the stores
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(tempty0 + 8 * buf);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) bw[j * 32 + lane] = __uint_as_float(send_u[j]);
+                    named_sync(1 + wp, 64);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const float other = br[j * 32 + lane];
+                        const float mine = __uint_as_float(keep_u[j]);
+                        patch[j * 32 + lane] = __float2bfloat16_rn(is_up ? swiglu(other, mine) : swiglu(mine, other));
+                    }
+                    __syncwarp();
+                    const int cb = c0 + (is_up ? 32 : 0);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int r = prow + 8 * i;
+                        const uint4 val = *reinterpret_cast<const uint4 *>(patch + r * 32 + pch * 8);
+                        if (f_ok && cb + r < it.n)
+                            *reinterpret_cast<uint4 *>(out + (size_t)(it.pos0 + cb + r) * out_ld + f0 + pch * 8) = val;
+                    }
+                    named_sync(1 + wp, 64);  // the partner has read this step's values before the next step overwrites them
+                }
+            } else {
+                const int row0 = 256 * it.mb + 128 * (int)rank + 32 * q;  // first of this warp's 32 output features
+                const bool r_ok = row0 < out_rows;
+                for (int c0 = 0; c0 < it.n; c0 += 32) {
+                    float v[32];
+                    tmem_ld32(t0 + c0, v);
+                    if (c0 + 32 >= it.n) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(tempty0 + 8 * buf);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) patch[j * 32 + lane] = __float2bfloat16_rn(v[j]);
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int r = prow + 8 * i;
+                        const uint4 val = *reinterpret_cast<const uint4 *>(patch + r * 32 + pch * 8);
+                        if (r_ok && c0 + r < it.n)
+                            *reinterpret_cast<uint4 *>(out + (size_t)(it.pos0 + c0 + r) * out_ld + row0 + pch * 8) = val;
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+        if (!ok && lane == 0) {
+            if (!*abort_flag) atomicExch(&meta[kMetaError], 13);
+            s_abort = 1;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // neither CTA leaves (or frees TMEM) while the other may still signal or read it
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
+template <int MODE, int HALF_MAX, int STAGES>
+constexpr int pair_smem_bytes() {
+    return STAGES * (kATileBytes + HALF_MAX * kRowBytes) + kPatchBytes + (MODE == 1 ? kXchgBytes : 0) + 1024;
+}
+
+template <int MODE, int HALF_MAX, int STAGES>
+bool set_smem_attr() {
+    return cudaFuncSetAttribute(expert_gemm_pair_kernel<MODE, HALF_MAX, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                pair_smem_bytes<MODE, HALF_MAX, STAGES>()) == cudaSuccess;
+}
+
+// small: at most 64 pair rows per expert (decode batches, T <= 64); big: up to 256 per tile
+constexpr int kSmallHalf = 32, kSmallStages1 = 9, kSmallStages2 = 10;
+constexpr int kBigHalf = 128, kBigStages1 = 6, kBigStages2 = 6;
+
+}  // namespace
+
+int init_pair_kernels(zeda_moe *h) {
+    const zeda_moe_config_t &c = h->cfg;
+    PairMaps *pm = static_cast<PairMaps *>(aligned_alloc(64, sizeof(PairMaps)));
+    if (!pm) { set_error("out of host memory"); return -1; }
+    const cuuint64_t E = c.n_real, d = c.d_model, He = c.d_expert;
+    const cuuint64_t rows = (cuuint64_t)c.max_tokens * c.top_k + kPairTileM;
+    bool ok = true;
+    {
+        // a 5-D view of [N][2 He][d] that lets one box fetch 64 gate rows and the matching 64 up rows:
+        // (k, row in block, gate | up, block of 64 rows, expert)
+        const cuuint64_t dims[5] = {d, 64, 2, He / 64, E};
+        const cuuint64_t strides[4] = {d * 2, He * d * 2, 64 * d * 2, 2 * He * d * 2};
+        const cuuint32_t box[5] = {kBlockK, 64, 2, 1, 1};
+        ok = ok && encode_bf16_map(&pm->w_gate_up, h->w_gate_up, 5, dims, strides, box);
+    }
+    {
+        const cuuint64_t dims[3] = {He, d, E};
+        const cuuint64_t strides[2] = {He * 2, d * He * 2};
+        const cuuint32_t box[3] = {kBlockK, 128, 1};
+        ok = ok && encode_bf16_map(&pm->w_down, h->w_down, 3, dims, strides, box);
+    }
+    for (int i = 0; i < 4; ++i) {
+        const cuuint64_t dims[2] = {He, rows};
+        const cuuint64_t strides[1] = {He * 2};
+        const cuuint32_t box[2] = {kBlockK, (cuuint32_t)(128 >> i)};
+        ok = ok && encode_bf16_map(&pm->hmid.m[i], h->ws.hmid, 2, dims, strides, box);
+    }
+    ok = ok && set_smem_attr<1, kSmallHalf, kSmallStages1>() && set_smem_attr<2, kSmallHalf, kSmallStages2>() &&
+         set_smem_attr<1, kBigHalf, kBigStages1>() && set_smem_attr<2, kBigHalf, kBigStages2>();
+    if (!ok) {
+        free(pm);
+        if (zeda_last_error()[0] == 0) set_error("pair kernel set-up failed: %s", cudaGetErrorString(cudaGetLastError()));
+        return -1;
+    }
+    h->pmaps = pm;
+    return 0;
+}
+
+int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s) {
+    const zeda_moe_config_t &c = h->cfg;
+    const Workspace &ws = h->ws;
+    const PairMaps *pm = static_cast<const PairMaps *>(h->pmaps);
+    const int m_blocks = (c.d_expert + 127) / 128;
+    const int grid = (h->sm_count / 2) * 2;
+    if (T <= 2 * kSmallHalf)
+        expert_gemm_pair_kernel<1, kSmallHalf, kSmallStages1><<<grid, kThreadsGather, pair_smem_bytes<1, kSmallHalf, kSmallStages1>(), s>>>(
+            pm->w_gate_up, pm->hmid, x, c.d_model, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
+            ws.meta, c.d_model, c.d_expert, m_blocks, ws.hmid, c.d_expert);
+    else
+        expert_gemm_pair_kernel<1, kBigHalf, kBigStages1><<<grid, kThreadsGather, pair_smem_bytes<1, kBigHalf, kBigStages1>(), s>>>(
+            pm->w_gate_up, pm->hmid, x, c.d_model, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
+            ws.meta, c.d_model, c.d_expert, m_blocks, ws.hmid, c.d_expert);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+int launch_experts_gemm2_pair(const zeda_moe *h, int T, cudaStream_t s) {
+    const zeda_moe_config_t &c = h->cfg;
+    const Workspace &ws = h->ws;
+    const PairMaps *pm = static_cast<const PairMaps *>(h->pmaps);
+    const int m_blocks = (c.d_model + 255) / 256;
+    const int grid = (h->sm_count / 2) * 2;
+    if (T <= 2 * kSmallHalf)
+        expert_gemm_pair_kernel<2, kSmallHalf, kSmallStages2><<<grid, kThreads, pair_smem_bytes<2, kSmallHalf, kSmallStages2>(), s>>>(
+            pm->w_down, pm->hmid, nullptr, 0, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
+            ws.meta, c.d_expert, c.d_model, m_blocks, ws.obuf, c.d_model);
+    else
+        expert_gemm_pair_kernel<2, kBigHalf, kBigStages2><<<grid, kThreads, pair_smem_bytes<2, kBigHalf, kBigStages2>(), s>>>(
+            pm->w_down, pm->hmid, nullptr, 0, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
+            ws.meta, c.d_expert, c.d_model, m_blocks, ws.obuf, c.d_model);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
+
+}  // namespace zeda

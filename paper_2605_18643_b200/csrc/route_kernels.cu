@@ -183,6 +183,7 @@ struct ScanShared {
     int32_t off[kMaxCand + 1];
     int32_t chunk[kMaxCand + 1];
     int32_t tile[kMaxCand + 1];
+    int32_t ptile[kMaxCand + 1];
 };
 
 // From per-expert pair counts in sh.cnt: exclusive offsets, P, U, and the work lists of the expert
@@ -190,33 +191,36 @@ struct ScanShared {
 __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, int total_slots,
                                                    int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
                                                    int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
-                                                   int32_t *__restrict__ chunk_expert, int32_t *__restrict__ chunk_row0,
-                                                   int32_t *__restrict__ tile_expert, int32_t *__restrict__ tile_row0) {
+                                                   const WorkLists &wl) {
     const int e = threadIdx.x;
     if (threadIdx.x < 32) {
         // warp 0 scans the three per-expert sequences in steps of 32 with shuffle prefix sums
-        int base_off = 0, base_chunk = 0, base_tile = 0, active = 0, max_rows = 0;
+        int base_off = 0, base_chunk = 0, base_tile = 0, base_ptile = 0, active = 0, max_rows = 0;
         for (int e0 = 0; e0 < n_real; e0 += 32) {
             const int i = e0 + threadIdx.x;
             const int c = (i < n_real) ? sh.cnt[i] : 0;
             const int ch = (c + kChunkRows - 1) / kChunkRows;
             const int tl = (c + kTileM - 1) / kTileM;
-            int so = c, sc = ch, st = tl;
+            const int pt = (c + kPairTileM - 1) / kPairTileM;
+            int so = c, sc = ch, st = tl, sp = pt;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const int a = __shfl_up_sync(kFull, so, o);
                 const int b = __shfl_up_sync(kFull, sc, o);
                 const int g = __shfl_up_sync(kFull, st, o);
-                if ((int)threadIdx.x >= o) { so += a; sc += b; st += g; }
+                const int q = __shfl_up_sync(kFull, sp, o);
+                if ((int)threadIdx.x >= o) { so += a; sc += b; st += g; sp += q; }
             }
             if (i < n_real) {
                 sh.off[i] = base_off + so - c;
                 sh.chunk[i] = base_chunk + sc - ch;
                 sh.tile[i] = base_tile + st - tl;
+                sh.ptile[i] = base_ptile + sp - pt;
             }
             base_off += __shfl_sync(kFull, so, 31);
             base_chunk += __shfl_sync(kFull, sc, 31);
             base_tile += __shfl_sync(kFull, st, 31);
+            base_ptile += __shfl_sync(kFull, sp, 31);
             active += __popc(__ballot_sync(kFull, c > 0));
             int mx = c;
 #pragma unroll
@@ -230,6 +234,7 @@ __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, i
             meta[kMetaZeroSlots] = total_slots - base_off;
             meta[kMetaChunks] = base_chunk;
             meta[kMetaTiles] = base_tile;
+            meta[kMetaPairTiles] = base_ptile;
             meta[kMetaMaxRows] = max_rows;
             if (n_pairs_out) *n_pairs_out = base_off;
         }
@@ -240,9 +245,11 @@ __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, i
         if (counts) counts[e] = c;
         offsets[e] = sh.off[e];
         int ci = sh.chunk[e];
-        for (int r = 0; r < c; r += kChunkRows, ++ci) { chunk_expert[ci] = e; chunk_row0[ci] = r; }
+        for (int r = 0; r < c; r += kChunkRows, ++ci) { wl.chunk_expert[ci] = e; wl.chunk_row0[ci] = r; }
         int ti = sh.tile[e];
-        for (int r = 0; r < c; r += kTileM, ++ti) { tile_expert[ti] = e; tile_row0[ti] = r; }
+        for (int r = 0; r < c; r += kTileM, ++ti) { wl.tile_expert[ti] = e; wl.tile_row0[ti] = r; }
+        int pi = sh.ptile[e];
+        for (int r = 0; r < c; r += kPairTileM, ++pi) { wl.ptile_expert[pi] = e; wl.ptile_row0[pi] = r; }
     }
     if (e == 0) offsets[n_real] = sh.off[n_real];
 }
@@ -250,9 +257,7 @@ __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, i
 __global__ void __launch_bounds__(512)
 expert_scan_kernel(int32_t *__restrict__ block_hist, int nblk, int n_real, int total_slots,
                    int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
-                   int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
-                   int32_t *__restrict__ chunk_expert, int32_t *__restrict__ chunk_row0,
-                   int32_t *__restrict__ tile_expert, int32_t *__restrict__ tile_row0) {
+                   int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta, const WorkLists wl) {
     __shared__ ScanShared sh;
     const int e = threadIdx.x;
     if (e < n_real) {
@@ -265,8 +270,7 @@ expert_scan_kernel(int32_t *__restrict__ block_hist, int nblk, int n_real, int t
         sh.cnt[e] = run;
     }
     __syncthreads();
-    finish_expert_scan(sh, n_real, total_slots, counts, offsets, n_pairs_out, meta, chunk_expert, chunk_row0,
-                       tile_expert, tile_row0);
+    finish_expert_scan(sh, n_real, total_slots, counts, offsets, n_pairs_out, meta, wl);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -287,8 +291,7 @@ __global__ void __cluster_dims__(kSmallCluster, 1, 1) __launch_bounds__(kSmallTh
 route_small_kernel(const float *__restrict__ logits, int T, int n_real, int n_cand, int K, int gate_mode,
                    int32_t *__restrict__ topk_idx, float *__restrict__ topk_w, int32_t *__restrict__ counts,
                    int32_t *__restrict__ offsets, int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
-                   int32_t *__restrict__ chunk_expert, int32_t *__restrict__ chunk_row0,
-                   int32_t *__restrict__ tile_expert, int32_t *__restrict__ tile_row0, int32_t *__restrict__ perm,
+                   const WorkLists wl, int32_t *__restrict__ perm,
                    int32_t *__restrict__ perm_user, int32_t *__restrict__ inv, int32_t *__restrict__ pair_token) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
@@ -320,8 +323,7 @@ route_small_kernel(const float *__restrict__ logits, int T, int n_real, int n_ca
         sh.cnt[threadIdx.x] = c;
     }
     __syncthreads();
-    finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, chunk_expert, chunk_row0, tile_expert,
-                       tile_row0);
+    finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, wl);
     for (int s = threadIdx.x; s < T * K; s += blockDim.x) {
         const int e = topk_idx[s], tk = s / K;
         int p = -1;
@@ -508,6 +510,7 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
     const Workspace &ws = h->ws;
     const int nblk = (T + kSortTokens - 1) / kSortTokens;
     int launches = 4;
+    const WorkLists wl = {ws.chunk_expert, ws.chunk_row0, ws.tile_expert, ws.tile_row0, ws.ptile_expert, ws.ptile_row0};
 #define ZEDA_RPL_DISPATCH(CALL)                        \
     do {                                               \
         if (n_cand <= 64) { CALL(2); }                 \
@@ -519,8 +522,7 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
 #define ZEDA_CALL_SMALL(R)                                                                                         \
     route_small_kernel<R><<<kSmallCluster, kSmallThreads, 0, s>>>(                                                 \
         logits, T, c.n_real, n_cand, K, c.gate_mode, ws.topk_idx, ws.topk_w, ws.counts, ws.offsets, out.n_pairs,   \
-        ws.meta, ws.chunk_expert, ws.chunk_row0, ws.tile_expert, ws.tile_row0, ws.perm, out.perm, ws.inv,          \
-        ws.pair_token)
+        ws.meta, wl, ws.perm, out.perm, ws.inv, ws.pair_token)
         ZEDA_RPL_DISPATCH(ZEDA_CALL_SMALL);
 #undef ZEDA_CALL_SMALL
         launches = 1;
@@ -531,7 +533,7 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
 #undef ZEDA_CALL_TOPK
         slot_hist_kernel<<<nblk, 256, sizeof(int32_t) * c.n_real, s>>>(ws.topk_idx, T, K, c.n_real, ws.block_hist);
         expert_scan_kernel<<<1, 512, 0, s>>>(ws.block_hist, nblk, c.n_real, T * K, ws.counts, ws.offsets, out.n_pairs,
-                                             ws.meta, ws.chunk_expert, ws.chunk_row0, ws.tile_expert, ws.tile_row0);
+                                             ws.meta, wl);
         slot_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * kPlaceWarps * c.n_real, s>>>(
             ws.topk_idx, T, K, c.n_real, ws.block_hist, ws.offsets, ws.perm, out.perm, ws.inv, ws.pair_token);
     }
@@ -580,6 +582,8 @@ struct StaticScratch {
     int32_t chunk_row0[kStaticLists];
     int32_t tile_expert[kStaticLists];
     int32_t tile_row0[kStaticLists];
+    int32_t ptile_expert[kStaticLists];
+    int32_t ptile_row0[kStaticLists];
     int32_t meta[kMetaCount];
 };
 
@@ -625,9 +629,10 @@ extern "C" zeda_status_t zeda_compact_static(const int32_t *topk_idx, int32_t T,
     if (e != cudaSuccess) { set_error("cudaMemsetAsync: %s", cudaGetErrorString(e)); return ZEDA_ERR_CUDA; }
     const int nblk = (T + kSortTokens - 1) / kSortTokens;
     slot_hist_kernel<<<nblk, 256, sizeof(int32_t) * n_real, s>>>(topk_idx, T, top_k, n_real, sc->block_hist);
+    const WorkLists wl = {sc->chunk_expert, sc->chunk_row0, sc->tile_expert, sc->tile_row0, sc->ptile_expert,
+                          sc->ptile_row0};
     expert_scan_kernel<<<1, 512, 0, s>>>(sc->block_hist, nblk, n_real, T * top_k, expert_counts, expert_offsets,
-                                         n_pairs, sc->meta, sc->chunk_expert, sc->chunk_row0, sc->tile_expert,
-                                         sc->tile_row0);
+                                         n_pairs, sc->meta, wl);
     slot_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * kPlaceWarps * n_real, s>>>(
         topk_idx, T, top_k, n_real, sc->block_hist, expert_offsets, perm, nullptr, sc->inv, sc->pair_token);
     e = cudaGetLastError();

@@ -69,13 +69,15 @@ size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int
     w.chunk_row0 = (int32_t *)take(chunks * 4);
     w.tile_expert = (int32_t *)take(tiles * 4);
     w.tile_row0 = (int32_t *)take(tiles * 4);
+    w.ptile_expert = (int32_t *)take(tiles * 4);
+    w.ptile_row0 = (int32_t *)take(tiles * 4);
     w.logits = (float *)take((size_t)c.max_tokens * n_cand * 4);
     w.stat_part = (float *)take(nblk_stats * 2 * n_cand * 4);
-    // pair buffers carry kTileM rows of slack so that a full tile may be stored past the last pair
-    w.hmid = (__nv_bfloat16 *)take((slots + kTileM) * c.d_expert * 2);
-    w.obuf = (__nv_bfloat16 *)take((slots + kTileM) * c.d_model * 2);
+    // pair buffers carry one tile of slack rows so that a full tile may be read past the last pair
+    w.hmid = (__nv_bfloat16 *)take((slots + kPairTileM) * c.d_expert * 2);
+    w.obuf = (__nv_bfloat16 *)take((slots + kPairTileM) * c.d_model * 2);
     w.router_split = (__nv_bfloat16 *)take((size_t)3 * router_split_pad((int)n_cand) * c.d_model * 2);
-    w.x_sorted = (__nv_bfloat16 *)take((slots + kTileM) * c.d_model * 2);
+    w.x_sorted = (__nv_bfloat16 *)take((slots + kPairTileM) * c.d_model * 2);
     w.x_stage = (__nv_bfloat16 *)take((size_t)c.max_tokens * c.d_model * 2);
     w.y_stage = (__nv_bfloat16 *)take((size_t)c.max_tokens * c.d_model * 2);
     if (ws) *ws = w;
@@ -128,17 +130,18 @@ zeda_status_t forward_device(zeda_moe_t *h, const __nv_bfloat16 *x, int T, __nv_
     if (r < 0) return cuda_fail("routing launch", cudaGetLastError());
     n += r;
     mark(2);
-    const bool tile = !(h->cfg.flags & ZEDA_FLAG_FORCE_STREAM_EXPERTS);
+    const bool stream = (h->cfg.flags & ZEDA_FLAG_FORCE_STREAM_EXPERTS) != 0;
+    const bool tile = (h->cfg.flags & ZEDA_FLAG_FORCE_TILE_EXPERTS) != 0;
     if (tile) {
         r = launch_gather_rows(h, x, T, s);
         if (r < 0) return cuda_fail("row gather launch", cudaGetLastError());
         n += r;
     }
-    r = tile ? launch_experts_gemm1_tile(h, T, s) : launch_experts_gemm1(h, x, T, s);
+    r = stream ? launch_experts_gemm1(h, x, T, s) : tile ? launch_experts_gemm1_tile(h, T, s) : launch_experts_gemm1_pair(h, x, T, s);
     if (r < 0) return cuda_fail("expert GEMM1 launch", cudaGetLastError());
     n += r;
     mark(3);
-    r = tile ? launch_experts_gemm2_tile(h, T, s) : launch_experts_gemm2(h, T, s);
+    r = stream ? launch_experts_gemm2(h, T, s) : tile ? launch_experts_gemm2_tile(h, T, s) : launch_experts_gemm2_pair(h, T, s);
     if (r < 0) return cuda_fail("expert GEMM2 launch", cudaGetLastError());
     n += r;
     mark(4);
@@ -203,6 +206,7 @@ zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_
     h->sm_count = prop.multiProcessorCount;
     h->last_launches = 0;
     h->tmaps = nullptr;
+    h->pmaps = nullptr;
     h->router_maps = nullptr;
     h->profiling = false;
     h->profiled_last = false;
@@ -210,8 +214,10 @@ zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_
     carve(*cfg, static_cast<unsigned char *>(workspace), &h->ws, &h->max_chunks, &h->max_tiles);
     if (init_route_kernels(h) < 0) { delete h; return cuda_fail("kernel set-up", cudaGetLastError()); }
     if (init_tile_kernels(h) < 0) { delete h; return ZEDA_ERR_CUDA; }
+    if (init_pair_kernels(h) < 0) { free(h->tmaps); delete h; return ZEDA_ERR_CUDA; }
     if (init_router_tile(h) < 0) {
         if (h->tmaps) free(h->tmaps);
+        if (h->pmaps) free(h->pmaps);
         delete h;
         return cuda_fail("router set-up", cudaGetLastError());
     }
@@ -358,6 +364,7 @@ zeda_status_t zeda_moe_destroy(zeda_moe_t *h) {
     }
     for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
     if (h->tmaps) free(h->tmaps);
+    if (h->pmaps) free(h->pmaps);
     if (h->router_maps) free(h->router_maps);
     delete h;
     return st;

@@ -13,7 +13,8 @@ constexpr int kMaxCand = 512;       // N + N_Z limit (16 logits per lane in the 
 constexpr int kMaxTopK = 16;
 constexpr int kSortTokens = 128;    // tokens per CTA in the counting sort (histogram / placement)
 constexpr int kChunkRows = 32;      // pair rows per work chunk of the streaming expert kernels
-constexpr int kTileM = 128;         // pair rows per tile of the tcgen05 expert kernels
+constexpr int kTileM = 128;         // pair rows per tile of the single-CTA tcgen05 expert kernels
+constexpr int kPairTileM = 256;     // pair rows per tile of the CTA-pair tcgen05 expert kernels
 
 // Device-resident counters of one call.
 enum MetaSlot {
@@ -24,6 +25,7 @@ enum MetaSlot {
     kMetaTiles = 4,      // M tiles for the tile kernels
     kMetaError = 5,      // sticky error word written by bounded device waits
     kMetaMaxRows = 6,    // largest per-expert pair count
+    kMetaPairTiles = 7,  // tiles for the CTA-pair kernels
     kMetaCount = 16
 };
 
@@ -41,6 +43,8 @@ struct Workspace {
     int32_t *chunk_row0;   // [maxChunks]
     int32_t *tile_expert;  // [maxTiles]
     int32_t *tile_row0;    // [maxTiles]
+    int32_t *ptile_expert; // [maxTiles] tiles of kPairTileM rows
+    int32_t *ptile_row0;   // [maxTiles]
     float *logits;         // [maxT*(N+N_Z)]
     float *stat_part;      // [nblk_stats * 2 * (N+N_Z)]
     __nv_bfloat16 *hmid;   // [maxT*K, He]
@@ -49,6 +53,12 @@ struct Workspace {
     __nv_bfloat16 *x_sorted; // [maxT*K, d] x rows in pair order (tile path)
     __nv_bfloat16 *x_stage;// [maxT, d]
     __nv_bfloat16 *y_stage;// [maxT, d]
+};
+
+struct WorkLists {  // device-side work lists written by the expert scan
+    int32_t *chunk_expert, *chunk_row0;  // chunks of kChunkRows pair rows
+    int32_t *tile_expert, *tile_row0;    // tiles of kTileM pair rows
+    int32_t *ptile_expert, *ptile_row0;  // tiles of kPairTileM pair rows
 };
 
 struct RouteOut {  // where one routing pass writes (user buffers or workspace)
@@ -74,6 +84,7 @@ struct zeda_moe {
     int max_tiles;
     int last_launches;
     void *tmaps;  // host-side tensor maps of the tile path (owned)
+    void *pmaps;  // host-side tensor maps of the CTA-pair path (owned)
     void *router_maps;  // host-side tensor map of the split router weights (owned)
     bool profiling;
     bool profiled_last;
@@ -97,6 +108,9 @@ int launch_router_logits_tile(const zeda_moe *h, const __nv_bfloat16 *x, int T, 
 int launch_gather_rows(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
 int launch_experts_gemm1_tile(const zeda_moe *h, int T, cudaStream_t s);
 int launch_experts_gemm2_tile(const zeda_moe *h, int T, cudaStream_t s);
+int init_pair_kernels(zeda_moe *h);
+int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
+int launch_experts_gemm2_pair(const zeda_moe *h, int T, cudaStream_t s);
 int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s);
 
 void set_error(const char *fmt, ...);
