@@ -83,7 +83,7 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "--id=%d" % self.index, "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                 "-lms", "20"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -166,6 +166,22 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+class L2Flush:
+    """Evicts the layer's data from L2 between timed steps: writes a 256 MiB buffer (twice the
+    126 MB L2), then reads a second one so that the lines left behind are clean.  (Dirty lines of
+    the written buffer would otherwise be written back during the timed step, which charges the
+    step with about 126 MB of DRAM writes that belong to the flush.)"""
+
+    def __init__(self, dev, nbytes=256 << 20):
+        self.w = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        self.r = torch.zeros(nbytes // 4, dtype=torch.float32, device=dev)
+        self.sink = None
+
+    def zero_(self):
+        self.w.zero_()
+        self.sink = self.r.sum()
+
+
 def time_forward(m, x, y, steps, warmup, flush, dist_barrier):
     """Per-step CUDA-event timing with an L2 flush (outside the event pairs) between steps."""
     for _ in range(warmup):
@@ -225,7 +241,7 @@ def main():
     m = zeda.from_workload(wl, dev)
     x = x_cpu.to(dev)
     y = torch.empty_like(x)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    flush = L2Flush(dev)
 
     clocks = ClockSampler(local_rank)
     clocks.start()
@@ -304,7 +320,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": workload_config(wl, args.workload, {
-                "P": P, "U": U, "l2": "256 MiB buffer written between timed steps (outside the event pairs)",
+                "P": P, "U": U, "l2": "256 MiB written, then 256 MiB read, between timed steps (outside the event pairs)",
                 "parallelism": "dp%d replicas, no collective" % world}),
             "clocks": clock_info,
             "e2e": {"value": world * wl.T * args.steps / e2e_s, "unit": UNIT,

@@ -110,25 +110,31 @@ __device__ __forceinline__ void topk_gate_token(const float *__restrict__ row, i
     }
     den = warp_sum(den);
 
-    unsigned taken = 0;  // bit r set: this lane's register r was already selected
+    // Selection on order-preserving integer keys (0 = not available), so that one warp-wide integer
+    // maximum finds the best logit and one integer minimum the lowest candidate id that holds it.
+    unsigned key[RPL];
+#pragma unroll
+    for (int r = 0; r < RPL; ++r) {
+        const unsigned u = __float_as_uint(v[r]);
+        key[r] = (r * 32 + lane < n_cand) ? ((u & 0x80000000u) ? ~u : (u | 0x80000000u)) : 0u;
+    }
     float my_p = 0.f;
     float sum_sel = 0.f, sum_real = 0.f;
     my_idx = -1;
     for (int k = 0; k < K; ++k) {
-        float bv = -INFINITY;
-        int bj = 0x7fffffff;
+        unsigned lm = key[0];
 #pragma unroll
-        for (int r = 0; r < RPL; ++r) {
-            const int j = r * 32 + lane;
-            if (j < n_cand && !((taken >> r) & 1u) && (v[r] > bv || bj == 0x7fffffff)) { bv = v[r]; bj = j; }
-        }
+        for (int r = 1; r < RPL; ++r) lm = max(lm, key[r]);
+        const unsigned gm = __reduce_max_sync(kFull, lm);
+        int cand = 0x7fffffff;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(kFull, bv, o);
-            const int oj = __shfl_xor_sync(kFull, bj, o);
-            if (oj != 0x7fffffff && (bj == 0x7fffffff || ov > bv || (ov == bv && oj < bj))) { bv = ov; bj = oj; }
-        }
-        if ((bj & 31) == lane) taken |= 1u << (bj >> 5);
+        for (int r = RPL - 1; r >= 0; --r)
+            if (key[r] == gm) cand = r * 32 + lane;  // ends on this lane's lowest id with that logit
+        const int bj = __reduce_min_sync(kFull, cand);
+#pragma unroll
+        for (int r = 0; r < RPL; ++r)
+            if (r * 32 + lane == bj) key[r] = 0u;
+        const float bv = __uint_as_float((gm & 0x80000000u) ? (gm & 0x7fffffffu) : ~gm);
         const float p = expf(bv - m) / den;
         sum_sel += p;
         if (bj < n_real) sum_real += p;
@@ -178,6 +184,8 @@ slot_hist_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real,
 // Counting sort, pass 2 (one CTA): column-wise exclusive scan over the CTA histograms, expert
 // counts, exclusive offsets, P, U, and the work lists of the expert kernels.
 // ---------------------------------------------------------------------------------------------
+constexpr int kScanSlabInts = 8192;  // 32 KB of CTA histograms per slab of the expert scan
+
 struct ScanShared {
     int32_t cnt[kMaxCand];
     int32_t off[kMaxCand + 1];
@@ -191,8 +199,7 @@ struct ScanShared {
 __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, int total_slots,
                                                    int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
                                                    int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
-                                                   const WorkLists &wl) {
-    const int e = threadIdx.x;
+                                                   const WorkLists &wl, bool write_global = true) {
     if (threadIdx.x < 32) {
         // warp 0 scans the three per-expert sequences in steps of 32 with shuffle prefix sums
         int base_off = 0, base_chunk = 0, base_tile = 0, base_ptile = 0, active = 0, max_rows = 0;
@@ -229,6 +236,11 @@ __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, i
         }
         if (threadIdx.x == 0) {
             sh.off[n_real] = base_off;
+            sh.chunk[n_real] = base_chunk;
+            sh.tile[n_real] = base_tile;
+            sh.ptile[n_real] = base_ptile;
+        }
+        if (threadIdx.x == 0 && write_global) {
             meta[kMetaPairs] = base_off;
             meta[kMetaActive] = active;
             meta[kMetaZeroSlots] = total_slots - base_off;
@@ -240,18 +252,28 @@ __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, i
         }
     }
     __syncthreads();
-    if (e < n_real) {
-        const int c = sh.cnt[e];
-        if (counts) counts[e] = c;
+    if (!write_global) return;  // (uniform over the CTA)
+    for (int e = threadIdx.x; e < n_real; e += blockDim.x) {
+        if (counts) counts[e] = sh.cnt[e];
         offsets[e] = sh.off[e];
-        int ci = sh.chunk[e];
-        for (int r = 0; r < c; r += kChunkRows, ++ci) { wl.chunk_expert[ci] = e; wl.chunk_row0[ci] = r; }
-        int ti = sh.tile[e];
-        for (int r = 0; r < c; r += kTileM, ++ti) { wl.tile_expert[ti] = e; wl.tile_row0[ti] = r; }
-        int pi = sh.ptile[e];
-        for (int r = 0; r < c; r += kPairTileM, ++pi) { wl.ptile_expert[pi] = e; wl.ptile_row0[pi] = r; }
     }
-    if (e == 0) offsets[n_real] = sh.off[n_real];
+    if (threadIdx.x == 0) offsets[n_real] = sh.off[n_real];
+    // work lists: entry i belongs to the expert whose first-entry index is the last one <= i
+    auto fill = [&](const int32_t *first, int rows, int32_t *list_expert, int32_t *list_row0) {
+        const int total = first[n_real];
+        for (int i = threadIdx.x; i < total; i += blockDim.x) {
+            int lo = 0, hi = n_real;  // invariant: first[lo] <= i < first[hi]
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (first[mid] <= i) lo = mid; else hi = mid;
+            }
+            list_expert[i] = lo;
+            list_row0[i] = (i - first[lo]) * rows;
+        }
+    };
+    fill(sh.chunk, kChunkRows, wl.chunk_expert, wl.chunk_row0);
+    fill(sh.tile, kTileM, wl.tile_expert, wl.tile_row0);
+    fill(sh.ptile, kPairTileM, wl.ptile_expert, wl.ptile_row0);
 }
 
 __global__ void __launch_bounds__(512)
@@ -259,16 +281,31 @@ expert_scan_kernel(int32_t *__restrict__ block_hist, int nblk, int n_real, int t
                    int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
                    int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta, const WorkLists wl) {
     __shared__ ScanShared sh;
+    // Exclusive scan of every expert column over the CTA histograms.  The histograms are staged in
+    // shared memory slab by slab with independent coalesced loads (a load-scan-store loop straight
+    // on global memory is a chain of dependent L2 round trips), scanned by one thread per expert,
+    // and written back coalesced.
+    __shared__ int32_t slab[kScanSlabInts];
+    const int slab_blocks = max(1, kScanSlabInts / n_real);
     const int e = threadIdx.x;
-    if (e < n_real) {
-        int run = 0;
-        for (int b = 0; b < nblk; ++b) {
-            const int c = block_hist[(size_t)b * n_real + e];
-            block_hist[(size_t)b * n_real + e] = run;  // pairs of expert e in earlier CTAs
-            run += c;
+    int run = 0;
+    for (int b0 = 0; b0 < nblk; b0 += slab_blocks) {
+        const int nb = min(slab_blocks, nblk - b0);
+        int32_t *g = block_hist + (size_t)b0 * n_real;
+        for (int i = threadIdx.x; i < nb * n_real; i += blockDim.x) slab[i] = g[i];
+        __syncthreads();
+        if (e < n_real) {
+            for (int b = 0; b < nb; ++b) {
+                const int c = slab[b * n_real + e];
+                slab[b * n_real + e] = run;  // pairs of expert e in earlier CTAs
+                run += c;
+            }
         }
-        sh.cnt[e] = run;
+        __syncthreads();
+        for (int i = threadIdx.x; i < nb * n_real; i += blockDim.x) g[i] = slab[i];
+        __syncthreads();
     }
+    if (e < n_real) sh.cnt[e] = run;
     __syncthreads();
     finish_expert_scan(sh, n_real, total_slots, counts, offsets, n_pairs_out, meta, wl);
 }
@@ -346,6 +383,7 @@ route_small_kernel(const float *__restrict__ logits, int T, int n_real, int n_ca
 // memory.  No atomics decide a position, so the order is (expert, token) ascending every run.
 // ---------------------------------------------------------------------------------------------
 constexpr int kPlaceWarps = 8;
+constexpr int kFoldMaxBlocks = 256;  // up to this many CTA histograms the placement CTAs scan them themselves
 
 __global__ void __launch_bounds__(kPlaceWarps * 32)
 slot_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real,
@@ -375,6 +413,81 @@ slot_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real
     // turn counts into start positions: global offset + earlier CTAs + earlier warps
     for (int e = threadIdx.x; e < n_real; e += blockDim.x) {
         int run = offsets[e] + block_base[(size_t)blockIdx.x * n_real + e];
+        for (int w = 0; w < kPlaceWarps; ++w) {
+            const int c = pos[w * n_real + e];
+            pos[w * n_real + e] = run;
+            run += c;
+        }
+    }
+    __syncthreads();
+    for (int s = w0 + lane; s - lane < w1; s += 32) {
+        int e = (s < w1) ? topk_idx[s] : -1;
+        const bool in_range = s < w1;
+        if (e >= n_real) e = -1;
+        const unsigned grp = __match_any_sync(kFull, e);
+        int p = -1;
+        if (e >= 0) p = mine[e] + __popc(grp & lt);
+        __syncwarp();
+        if (e >= 0 && (grp & lt) == 0) mine[e] += __popc(grp);
+        __syncwarp();
+        if (in_range) {
+            inv[s] = p;
+            if (p >= 0) {
+                perm[p] = s;
+                if (perm_user) perm_user[p] = s;
+                pair_token[p] = s / K;
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Counting sort, passes 2 + 3 in one launch (used while the CTA histograms are few): every CTA
+// sums the histogram columns itself (pairs of each expert in earlier CTAs, and in all CTAs), scans
+// the expert totals, and places its slots as above.  CTA 0 also publishes counts, offsets, the
+// counters and the work lists.  Saves a launch and the single-CTA scan between two short kernels.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kPlaceWarps * 32)
+slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real, int nblk,
+                       const int32_t *__restrict__ block_hist, int32_t *__restrict__ counts,
+                       int32_t *__restrict__ offsets, int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
+                       const WorkLists wl, int32_t *__restrict__ perm, int32_t *__restrict__ perm_user,
+                       int32_t *__restrict__ inv, int32_t *__restrict__ pair_token) {
+    __shared__ ScanShared sh;
+    extern __shared__ int32_t pos[];       // [kPlaceWarps][n_real], then base[n_real]
+    int32_t *base = pos + kPlaceWarps * n_real;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int i = threadIdx.x; i < kPlaceWarps * n_real; i += blockDim.x) pos[i] = 0;
+    for (int e = threadIdx.x; e < n_real; e += blockDim.x) {
+        int before = 0, total = 0;
+        for (int b = 0; b < nblk; ++b) {
+            const int c = __ldg(block_hist + (size_t)b * n_real + e);
+            total += c;
+            if (b < (int)blockIdx.x) before += c;
+        }
+        base[e] = before;
+        sh.cnt[e] = total;
+    }
+    __syncthreads();
+    finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, wl, blockIdx.x == 0);
+    __syncthreads();
+    const int s0 = blockIdx.x * kSortTokens * K;
+    const int s1 = min(T * K, s0 + kSortTokens * K);
+    const int per_warp = ((kSortTokens * K + kPlaceWarps - 1) / kPlaceWarps + 31) / 32 * 32;
+    const int w0 = s0 + warp * per_warp;
+    const int w1 = min(s1, w0 + per_warp);
+    int32_t *mine = pos + warp * n_real;
+    const unsigned lt = (1u << lane) - 1u;
+    for (int s = w0 + lane; s - lane < w1; s += 32) {
+        int e = (s < w1) ? topk_idx[s] : -1;
+        if (e >= n_real) e = -1;
+        const unsigned grp = __match_any_sync(kFull, e);
+        if (e >= 0 && (grp & lt) == 0) mine[e] += __popc(grp);
+        __syncwarp();
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < n_real; e += blockDim.x) {
+        int run = sh.off[e] + base[e];
         for (int w = 0; w < kPlaceWarps; ++w) {
             const int c = pos[w * n_real + e];
             pos[w * n_real + e] = run;
@@ -532,10 +645,17 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
         ZEDA_RPL_DISPATCH(ZEDA_CALL_TOPK);
 #undef ZEDA_CALL_TOPK
         slot_hist_kernel<<<nblk, 256, sizeof(int32_t) * c.n_real, s>>>(ws.topk_idx, T, K, c.n_real, ws.block_hist);
-        expert_scan_kernel<<<1, 512, 0, s>>>(ws.block_hist, nblk, c.n_real, T * K, ws.counts, ws.offsets, out.n_pairs,
-                                             ws.meta, wl);
-        slot_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * kPlaceWarps * c.n_real, s>>>(
-            ws.topk_idx, T, K, c.n_real, ws.block_hist, ws.offsets, ws.perm, out.perm, ws.inv, ws.pair_token);
+        if (nblk <= kFoldMaxBlocks) {
+            slot_scan_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * (kPlaceWarps + 1) * c.n_real, s>>>(
+                ws.topk_idx, T, K, c.n_real, nblk, ws.block_hist, ws.counts, ws.offsets, out.n_pairs, ws.meta, wl,
+                ws.perm, out.perm, ws.inv, ws.pair_token);
+            launches = 3;
+        } else {
+            expert_scan_kernel<<<1, 512, 0, s>>>(ws.block_hist, nblk, c.n_real, T * K, ws.counts, ws.offsets,
+                                                 out.n_pairs, ws.meta, wl);
+            slot_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * kPlaceWarps * c.n_real, s>>>(
+                ws.topk_idx, T, K, c.n_real, ws.block_hist, ws.offsets, ws.perm, out.perm, ws.inv, ws.pair_token);
+        }
     }
     if (cudaGetLastError() != cudaSuccess) return -1;
     // copies for a caller that asked for the routing itself
