@@ -78,7 +78,9 @@ typedef struct {
 enum {
     ZEDA_FLAG_NONE = 0,
     ZEDA_FLAG_FORCE_STREAM_EXPERTS = 1, /* always use the weight-streaming expert kernels */
-    ZEDA_FLAG_FORCE_TILE_EXPERTS = 2    /* always use the tcgen05 tile kernels */
+    ZEDA_FLAG_FORCE_TILE_EXPERTS = 2,   /* always use the single-CTA tcgen05 tile kernels */
+    ZEDA_FLAG_NO_DEPENDENT_LAUNCH = 4   /* launch every kernel fully stream-ordered (no programmatic
+                                           dependent launch between the kernels of a call) */
 };
 
 /* Device workspace the handle needs for the given configuration (bytes, multiple of 256);

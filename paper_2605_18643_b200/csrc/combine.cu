@@ -22,6 +22,8 @@ __global__ void __launch_bounds__(256)
 combine_kernel(const __nv_bfloat16 *__restrict__ obuf, const int32_t *__restrict__ inv,
                const float *__restrict__ topk_w, const __nv_bfloat16 *__restrict__ x, int K, int d,
                int copy_experts, __nv_bfloat16 *__restrict__ y) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int t = blockIdx.x;
     __shared__ int32_t s_pos[kMaxTopK];
     __shared__ float s_w[kMaxTopK];
@@ -67,9 +69,9 @@ int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat
     const int chunks = c.d_model / 8;
     const int threads = (T >= 1024 && chunks >= 256) ? 256 : (T >= 256 && chunks >= 128 ? 128 : 64);
     const int gy = (chunks + threads - 1) / threads;
-    combine_kernel<<<dim3(T, gy), threads, 0, s>>>(h->ws.obuf, h->ws.inv, h->ws.topk_w, x, c.top_k, c.d_model,
-                                         c.expert_kind == ZEDA_EXPERT_COPY, y);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    const cudaError_t e = launch_kernel(h->pdl, combine_kernel, dim3(T, gy), dim3(threads), 0, s, h->ws.obuf, h->ws.inv,
+                                        h->ws.topk_w, x, c.top_k, c.d_model, (int)(c.expert_kind == ZEDA_EXPERT_COPY), y);
+    return e == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace zeda

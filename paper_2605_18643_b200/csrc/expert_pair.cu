@@ -88,6 +88,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                         int32_t *__restrict__ meta, int kdim, int out_rows, int m_blocks,
                         __nv_bfloat16 *__restrict__ out, int out_ld) {
     constexpr int kStageBytes = kATileBytes + HALF_MAX * kRowBytes;
+    pdl_launch_dependents();
     extern __shared__ __align__(1024) unsigned char pair_smem[];
     __shared__ __align__(8) unsigned long long bars[3 * STAGES + 4];
     __shared__ uint32_t s_tmem_base;
@@ -127,6 +128,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
     volatile int *abort_flag = &s_abort;
+    pdl_wait();  // everything above is local set-up; the routing results and activations are read below
 
     const long long n_items = (long long)meta[kMetaPairTiles] * m_blocks;
     const int k_steps = kdim / kBlockK;
@@ -444,15 +446,16 @@ int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, int T, 
     const PairMaps *pm = static_cast<const PairMaps *>(h->pmaps);
     const int m_blocks = (c.d_expert + 127) / 128;
     const int grid = (h->sm_count / 2) * 2;
+    cudaError_t e;
     if (T <= 2 * kSmallHalf)
-        expert_gemm_pair_kernel<1, kSmallHalf, kSmallStages1><<<grid, kThreadsGather, pair_smem_bytes<1, kSmallHalf, kSmallStages1>(), s>>>(
+        e = launch_kernel(h->pdl, expert_gemm_pair_kernel<1, kSmallHalf, kSmallStages1>, dim3(grid), dim3(kThreadsGather), pair_smem_bytes<1, kSmallHalf, kSmallStages1>(), s,
             pm->w_gate_up, pm->hmid, x, c.d_model, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
             ws.meta, c.d_model, c.d_expert, m_blocks, ws.hmid, c.d_expert);
     else
-        expert_gemm_pair_kernel<1, kBigHalf, kBigStages1><<<grid, kThreadsGather, pair_smem_bytes<1, kBigHalf, kBigStages1>(), s>>>(
+        e = launch_kernel(h->pdl, expert_gemm_pair_kernel<1, kBigHalf, kBigStages1>, dim3(grid), dim3(kThreadsGather), pair_smem_bytes<1, kBigHalf, kBigStages1>(), s,
             pm->w_gate_up, pm->hmid, x, c.d_model, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
             ws.meta, c.d_model, c.d_expert, m_blocks, ws.hmid, c.d_expert);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    return e == cudaSuccess ? 1 : -1;
 }
 
 int launch_experts_gemm2_pair(const zeda_moe *h, int T, cudaStream_t s) {
@@ -461,15 +464,16 @@ int launch_experts_gemm2_pair(const zeda_moe *h, int T, cudaStream_t s) {
     const PairMaps *pm = static_cast<const PairMaps *>(h->pmaps);
     const int m_blocks = (c.d_model + 255) / 256;
     const int grid = (h->sm_count / 2) * 2;
+    cudaError_t e;
     if (T <= 2 * kSmallHalf)
-        expert_gemm_pair_kernel<2, kSmallHalf, kSmallStages2><<<grid, kThreads, pair_smem_bytes<2, kSmallHalf, kSmallStages2>(), s>>>(
-            pm->w_down, pm->hmid, nullptr, 0, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
+        e = launch_kernel(h->pdl, expert_gemm_pair_kernel<2, kSmallHalf, kSmallStages2>, dim3(grid), dim3(kThreads), pair_smem_bytes<2, kSmallHalf, kSmallStages2>(), s,
+            pm->w_down, pm->hmid, (const __nv_bfloat16 *)nullptr, 0, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
             ws.meta, c.d_expert, c.d_model, m_blocks, ws.obuf, c.d_model);
     else
-        expert_gemm_pair_kernel<2, kBigHalf, kBigStages2><<<grid, kThreads, pair_smem_bytes<2, kBigHalf, kBigStages2>(), s>>>(
-            pm->w_down, pm->hmid, nullptr, 0, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
+        e = launch_kernel(h->pdl, expert_gemm_pair_kernel<2, kBigHalf, kBigStages2>, dim3(grid), dim3(kThreads), pair_smem_bytes<2, kBigHalf, kBigStages2>(), s,
+            pm->w_down, pm->hmid, (const __nv_bfloat16 *)nullptr, 0, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
             ws.meta, c.d_expert, c.d_model, m_blocks, ws.obuf, c.d_model);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    return e == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace zeda

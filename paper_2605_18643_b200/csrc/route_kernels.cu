@@ -28,6 +28,8 @@ __global__ void __launch_bounds__(256)
 router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ router_w,
                      const float *__restrict__ router_bias, int T, int d, int n_cand,
                      int cand_per_cta, float *__restrict__ logits) {
+    pdl_launch_dependents();
+    pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __nv_bfloat16 *xs = reinterpret_cast<__nv_bfloat16 *>(smem_raw);  // [kTok][d]
     const int t0 = blockIdx.x * kTok;
@@ -149,6 +151,8 @@ template <int RPL>
 __global__ void __launch_bounds__(256)
 topk_gate_kernel(const float *__restrict__ logits, int T, int n_real, int n_cand, int K, int gate_mode,
                  int32_t *__restrict__ topk_idx, float *__restrict__ topk_w) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t = blockIdx.x * (blockDim.x >> 5) + warp;
     if (t >= T) return;
@@ -167,6 +171,8 @@ topk_gate_kernel(const float *__restrict__ logits, int T, int n_real, int n_cand
 __global__ void __launch_bounds__(256)
 slot_hist_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real,
                  int32_t *__restrict__ block_hist) {
+    pdl_launch_dependents();
+    pdl_wait();
     extern __shared__ int32_t hist[];  // [n_real]
     for (int e = threadIdx.x; e < n_real; e += blockDim.x) hist[e] = 0;
     __syncthreads();
@@ -330,6 +336,8 @@ route_small_kernel(const float *__restrict__ logits, int T, int n_real, int n_ca
                    int32_t *__restrict__ offsets, int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
                    const WorkLists wl, int32_t *__restrict__ perm,
                    int32_t *__restrict__ perm_user, int32_t *__restrict__ inv, int32_t *__restrict__ pair_token) {
+    pdl_launch_dependents();
+    pdl_wait();
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ ScanShared sh;
@@ -453,6 +461,8 @@ slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n
                        int32_t *__restrict__ offsets, int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
                        const WorkLists wl, int32_t *__restrict__ perm, int32_t *__restrict__ perm_user,
                        int32_t *__restrict__ inv, int32_t *__restrict__ pair_token) {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ ScanShared sh;
     extern __shared__ int32_t pos[];       // [kPlaceWarps][n_real], then base[n_real]
     int32_t *base = pos + kPlaceWarps * n_real;
@@ -612,9 +622,9 @@ int launch_router_logits(const zeda_moe *h, const __nv_bfloat16 *x, int T, float
     if (splits > max_splits) splits = max_splits;
     const int per = (n_cand + splits - 1) / splits;
     const size_t smem = (size_t)kTok * d * sizeof(__nv_bfloat16);
-    router_logits_kernel<<<dim3(tiles, (n_cand + per - 1) / per), 256, smem, s>>>(
-        x, h->router_w, h->router_bias, T, d, n_cand, per, logits);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    const cudaError_t e = launch_kernel(h->pdl, router_logits_kernel, dim3(tiles, (n_cand + per - 1) / per), dim3(256), smem, s,
+                                        x, h->router_w, h->router_bias, T, d, n_cand, per, logits);
+    return e == cudaSuccess ? 1 : -1;
 }
 
 int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, const RouteOut &out, cudaStream_t s) {
@@ -633,7 +643,7 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
     } while (0)
     if (T <= kSmallTokens && c.n_real <= kSmallThreads) {
 #define ZEDA_CALL_SMALL(R)                                                                                         \
-    route_small_kernel<R><<<kSmallCluster, kSmallThreads, 0, s>>>(                                                 \
+    launch_kernel(h->pdl, route_small_kernel<R>, dim3(kSmallCluster), dim3(kSmallThreads), 0, s,                    \
         logits, T, c.n_real, n_cand, K, c.gate_mode, ws.topk_idx, ws.topk_w, ws.counts, ws.offsets, out.n_pairs,   \
         ws.meta, wl, ws.perm, out.perm, ws.inv, ws.pair_token)
         ZEDA_RPL_DISPATCH(ZEDA_CALL_SMALL);
@@ -641,14 +651,17 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
         launches = 1;
     } else {
 #define ZEDA_CALL_TOPK(R) \
-    topk_gate_kernel<R><<<(T + 7) / 8, 256, 0, s>>>(logits, T, c.n_real, n_cand, K, c.gate_mode, ws.topk_idx, ws.topk_w)
+    launch_kernel(h->pdl, topk_gate_kernel<R>, dim3((T + 7) / 8), dim3(256), 0, s, logits, T, c.n_real, n_cand, K, \
+                  c.gate_mode, ws.topk_idx, ws.topk_w)
         ZEDA_RPL_DISPATCH(ZEDA_CALL_TOPK);
 #undef ZEDA_CALL_TOPK
-        slot_hist_kernel<<<nblk, 256, sizeof(int32_t) * c.n_real, s>>>(ws.topk_idx, T, K, c.n_real, ws.block_hist);
+        launch_kernel(h->pdl, slot_hist_kernel, dim3(nblk), dim3(256), sizeof(int32_t) * c.n_real, s,
+                      (const int32_t *)ws.topk_idx, T, K, c.n_real, ws.block_hist);
         if (nblk <= kFoldMaxBlocks) {
-            slot_scan_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * (kPlaceWarps + 1) * c.n_real, s>>>(
-                ws.topk_idx, T, K, c.n_real, nblk, ws.block_hist, ws.counts, ws.offsets, out.n_pairs, ws.meta, wl,
-                ws.perm, out.perm, ws.inv, ws.pair_token);
+            launch_kernel(h->pdl, slot_scan_place_kernel, dim3(nblk), dim3(kPlaceWarps * 32),
+                          sizeof(int32_t) * (kPlaceWarps + 1) * c.n_real, s, (const int32_t *)ws.topk_idx, T, K, c.n_real,
+                          nblk, (const int32_t *)ws.block_hist, ws.counts, ws.offsets, out.n_pairs, ws.meta, wl, ws.perm,
+                          out.perm, ws.inv, ws.pair_token);
             launches = 3;
         } else {
             expert_scan_kernel<<<1, 512, 0, s>>>(ws.block_hist, nblk, c.n_real, T * K, ws.counts, ws.offsets,

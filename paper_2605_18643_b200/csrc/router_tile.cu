@@ -48,6 +48,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 router_logits_tile_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
                           const float *__restrict__ bias, int T, int n_cand, int m_tiles, int k_steps,
                           int32_t *__restrict__ meta, float *__restrict__ logits) {
+    pdl_launch_dependents();
     extern __shared__ __align__(1024) unsigned char router_smem[];
     __shared__ __align__(8) unsigned long long bars[2 * kStages + 2];
     __shared__ uint32_t s_tmem_base;
@@ -72,6 +73,7 @@ router_logits_tile_kernel(const __grid_constant__ CUtensorMap map_w, const __gri
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
     volatile int *abort_flag = &s_abort;
+    pdl_wait();
     const int tok_tiles = (T + kTokTile - 1) / kTokTile;
     const int n_items = tok_tiles * m_tiles;
 
@@ -201,9 +203,10 @@ int launch_router_logits_tile(const zeda_moe *h, const __nv_bfloat16 *x, int T, 
     const int m_tiles = nc_pad / 128;
     const int n_items = (T + kTokTile - 1) / kTokTile * m_tiles;
     const int grid = n_items < h->sm_count ? n_items : h->sm_count;
-    router_logits_tile_kernel<<<grid, kThreads, kSmemBytes, s>>>(rm->w_split, map_x, h->router_bias, T, n_cand, m_tiles,
-                                                               c.d_model / kBlockK, h->ws.meta, logits);
-    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+    const cudaError_t e = launch_kernel(h->pdl, router_logits_tile_kernel, dim3(grid), dim3(kThreads), kSmemBytes, s,
+                                        rm->w_split, map_x, h->router_bias, T, n_cand, m_tiles, c.d_model / kBlockK,
+                                        h->ws.meta, logits);
+    return e == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace zeda

@@ -204,6 +204,7 @@ zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_
     h->w_gate_up = static_cast<const __nv_bfloat16 *>(w_gate_up);
     h->w_down = static_cast<const __nv_bfloat16 *>(w_down);
     h->sm_count = prop.multiProcessorCount;
+    h->pdl = !(cfg->flags & ZEDA_FLAG_NO_DEPENDENT_LAUNCH);
     h->last_launches = 0;
     h->tmaps = nullptr;
     h->pmaps = nullptr;

@@ -74,6 +74,7 @@ struct RouteOut {  // where one routing pass writes (user buffers or workspace)
 
 struct zeda_moe {
     zeda_moe_config_t cfg;
+    bool pdl;  // launch the forward kernels with programmatic stream serialization
     const float *router_w;
     const float *router_bias;
     const __nv_bfloat16 *w_gate_up;
@@ -114,5 +115,33 @@ int launch_experts_gemm2_pair(const zeda_moe *h, int T, cudaStream_t s);
 int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s);
 
 void set_error(const char *fmt, ...);
+
+// ---- programmatic dependent launch ------------------------------------------------------------
+// The kernels of one forward pass are launched back to back on one stream.  Launched with the
+// attribute below, a kernel may start (launch latency, barrier and TMEM set-up) while its
+// predecessor is still draining; it touches no global memory until pdl_wait() returns, which is
+// when the predecessor has completed and its writes are visible.  Each kernel calls
+// pdl_launch_dependents() first thing so that its successor is released as early as possible.
+// Without the attribute both calls do nothing.
+#if defined(__CUDACC__)
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                 Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
 
 }  // namespace zeda
