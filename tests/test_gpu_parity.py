@@ -280,3 +280,46 @@ def test_sweep_config_sampled(zeda, f):
     ids = sample_tokens(wl.T, 64, int(f * 100))
     err, (P, U, zs) = run_layer(zeda, wl, token_ids=ids, check_routing=False)
     assert abs(zs / (wl.T * wl.K) - f) < 0.02
+
+
+# ---------------------------------------------------------------------------------- kernel-path coverage
+
+def test_dependent_launch_flag_gives_identical_bits(zeda):
+    # the same kernels launched fully stream-ordered (flag 4) and with programmatic dependent launch
+    wl = inputs.tiny(seed=5, T=700)
+    dev = torch.device("cuda:0")
+    x = wl.x.to(dev)
+    outs = []
+    for flags in (0, 4):
+        m = zeda.from_workload(wl, dev, flags=flags)
+        for _ in range(3):  # back-to-back calls overlap the tail of one with the head of the next
+            y = m.forward(x)
+        torch.cuda.synchronize()
+        outs.append(y.view(torch.int16).clone())
+        m.close()
+    assert torch.equal(outs[0], outs[1])
+
+
+@pytest.mark.parametrize("d,He", [(320, 192), (64, 64), (576, 448)])
+def test_ragged_weight_row_blocks(zeda, d, He):
+    # d not a multiple of 256 and H_e not a multiple of 128: the last weight-row block of both
+    # expert GEMMs is partly (or, for one CTA of the pair, wholly) out of range
+    wl = inputs.tiny(seed=6, T=200, d=d, He=He)
+    run_layer(zeda, wl, token_ids=sample_tokens(200, 40, 3))
+
+
+def test_experts_with_many_tiles(zeda):
+    # few experts, many tokens: every expert spans several 256-row tiles plus a ragged one
+    wl = inputs.tiny(seed=7, T=3000, E=4, Z=2)
+    err, (P, U, zs) = run_layer(zeda, wl, token_ids=sample_tokens(3000, 48, 4))
+    assert U == 4 and P > 4 * 256
+
+
+def test_routing_with_many_sort_blocks(zeda):
+    # more than 256 blocks of 128 tokens: the counting sort takes its three-launch path
+    wl = inputs.tiny(seed=8, T=33000, d=64, He=64)
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev)
+    l, idx, w, counts, offsets, perm, P = oracle_route(wl)
+    check_route(m.route(wl.x.to(dev)), idx, w, counts, offsets, perm, P)
+    m.close()
