@@ -30,6 +30,9 @@ from paper_2605_18643_b200 import flops, inputs
 
 METRIC = "MoE-layer tokens/s"
 UNIT = "tokens/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (expert GEMM1),
+# from the ncu captures summarised under profiles/ (same workloads, same kernel build)
+NCU_TRAFFIC_BYTES = {"prefill": 621.5e6, "decode": 741.2e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -307,14 +310,21 @@ def main():
         g1_bytes = U * 2 * wl.He * wl.d * 2 + wl.T * wl.d * 2 + P * wl.He * 2
         g1_flops = 4 * P * wl.d * wl.He
         g1_s = stage[2] * 1e-3
-        hbm_bound = g1_bytes / hbm >= g1_flops / (peaks["bf16_tflops"] * 1e12)
+        # The kernel is timed by stage events inside the step, back to back with the other kernels:
+        # the tensor peak it is held against is the sustained one; the burst figure is given beside it.
+        burst = peaks["bf16_tflops"]
+        sustained = peaks.get("bf16_tflops_sustained", burst)
+        hbm_bound = g1_bytes / hbm >= g1_flops / (sustained * 1e12)
         if hbm_bound:
             roof = {"bound": "hbm", "achieved": g1_bytes / g1_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
         else:
-            roof = {"bound": "tensor", "achieved": g1_flops / g1_s / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+            roof = {"bound": "tensor", "achieved": g1_flops / g1_s / 1e12, "peak": sustained, "unit": "TFLOP/s",
+                    "peak_kind": "sustained (kernel timed inside the step)", "peak_burst": burst,
+                    "frac_of_burst": g1_flops / g1_s / 1e12 / burst}
         roof["frac"] = roof["achieved"] / roof["peak"]
-        roof.update(traffic=None, kernel="expert GEMM1 + SwiGLU", peak_source=peaks_kind,
-                    algorithmic_bytes=g1_bytes, algorithmic_flops=g1_flops, kernel_ms=stage[2])
+        roof.update(traffic=NCU_TRAFFIC_BYTES.get(args.workload), kernel="expert GEMM1 + SwiGLU (expert_gemm_pair_kernel<1,..>)",
+                    peak_source=peaks_kind, algorithmic_bytes=g1_bytes, algorithmic_flops=g1_flops, kernel_ms=stage[2])
+        t_roof_s, t_flop_s, _ = flops.layer_roofline_seconds(wl.T, wl.d, wl.He, n_cand, P, U, sustained * 1e12, hbm)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -329,7 +339,9 @@ def main():
             "gpu_launches": launches * args.steps,
             "roofline": roof,
             "layer_roofline": {"t_roof_us": t_roof * 1e6, "t_flop_us": t_flop * 1e6, "t_hbm_us": t_mem * 1e6,
-                               "frac": t_roof / (ms_per_step * 1e-3), "peak_source": peaks_kind},
+                               "frac": t_roof / (ms_per_step * 1e-3), "peak_source": peaks_kind,
+                               "t_flop_us_sustained": t_flop_s * 1e6, "t_roof_us_sustained": t_roof_s * 1e6,
+                               "frac_sustained": t_roof_s / (ms_per_step * 1e-3)},
             "stage_ms": {n: float(v) for n, v in zip(names, stage)},
         }
         if static:
