@@ -136,6 +136,16 @@ zeda_status_t zeda_moe_forward(zeda_moe_t *h, const void *x, int32_t T, void *y,
 zeda_status_t zeda_moe_forward_host(zeda_moe_t *h, const void *x_host, int32_t T, void *y_host,
                                     void *stream);
 
+/* Glue between stacked layers (the paper's models stack 48 such MoE layers, Section 4.2; the
+ * paper defines nothing between them, this is the layer-stack workload's device): in one pass
+ *   r <- bf16(r + y)                         residual stream, updated in place (y NULL: r is kept)
+ *   h  = r / sqrt(mean(r^2) + eps)           gain-free RMS normalisation, fp32 math, bf16 out
+ *   r  dev [T, d_model] bf16 (in/out)   y  dev [T, d_model] bf16 or NULL   h  dev [T, d_model] bf16
+ * Runs on the current device; needs no handle.  d_model: multiple of 64 in [64, 8192] (else
+ * ZEDA_ERR_UNSUPPORTED); pointers 16-byte aligned; h must not overlap r or y.  T = 0 touches nothing. */
+zeda_status_t zeda_residual_rmsnorm(void *r, const void *y, void *h, int32_t T, int32_t d_model, float eps,
+                                    void *stream);
+
 /* Routing statistics of the most recent zeda_route / zeda_moe_forward call on this handle
  * (Section 2.2, Eq. 4-6), computed on the device from that call's routing:
  *   f      dev [N+N_Z] fp32  share of tokens whose top-K set holds candidate i (f_i), or NULL

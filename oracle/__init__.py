@@ -155,3 +155,37 @@ def stats(logits_f32, topk_idx, n_real, n_zero, alpha=1.0, group_w=1.0):
                               ctypes.c_int(K), ctypes.c_double(alpha), ctypes.c_double(group_w),
                               _p(f), _p(pm), _p(out))
     return {"f": f, "P": pm, "r_ze": float(out[0]), "L_A": float(out[1]), "L_GA": float(out[2])}
+
+
+def _bf16_to_f64(bits):
+    return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def _f64_to_bf16_bits(v):
+    """Round-to-nearest-even of float64 values to bf16 bit patterns (via the exact float32 when the
+    value is one, else through the integer significand; inputs here are sums of two bf16 values,
+    which float64 holds exactly)."""
+    v = np.asarray(v, dtype=np.float64)
+    f = v.astype(np.float32)  # exact or correctly rounded once; see the callers' note
+    u = f.view(np.uint32).astype(np.uint64)
+    lsb = (u >> 16) & 1
+    r = (u + 0x7FFF + lsb) >> 16
+    return r.astype(np.uint16)
+
+
+def residual_rmsnorm(r_bits, y_bits=None, eps=1e-6):
+    """Glue between stacked MoE blocks (a device of the layer-stack workload, not part of the
+    paper's layer): r' = bf16(r + y) element by element (y may be None: r' = r), then the gain-free
+    RMS normalisation h = r' / sqrt(mean(r'^2) + eps) per row, in fp64.
+
+    Returns (r' as uint16 bit patterns, h as float64).  The sum of two bf16 values is exact in
+    float32 whenever their exponents differ by at most 16, and rounds back to the larger operand
+    otherwise, so rounding it through float32 and then to bf16 equals rounding the exact sum."""
+    r = _bf16_to_f64(r_bits)
+    if y_bits is not None:
+        r_new_bits = _f64_to_bf16_bits(r + _bf16_to_f64(y_bits))
+    else:
+        r_new_bits = np.ascontiguousarray(r_bits, dtype=np.uint16).copy()
+    rn = _bf16_to_f64(r_new_bits)
+    ms = np.mean(rn * rn, axis=-1, keepdims=True)
+    return r_new_bits, rn / np.sqrt(ms + eps)

@@ -24,7 +24,8 @@ FLAG_NONE, FLAG_FORCE_STREAM_EXPERTS, FLAG_FORCE_TILE_EXPERTS, FLAG_NO_DEPENDENT
 EXPORTS = (
     "zeda_moe_workspace_bytes", "zeda_moe_create", "zeda_route", "zeda_route_from_logits",
     "zeda_router_logits", "zeda_moe_forward", "zeda_moe_forward_host", "zeda_moe_stats",
-    "zeda_moe_last_counters", "zeda_moe_set_profiling", "zeda_moe_stage_ms", "zeda_compact_static", "zeda_moe_destroy", "zeda_last_error", "zeda_version",
+    "zeda_moe_last_counters", "zeda_moe_set_profiling", "zeda_moe_stage_ms", "zeda_residual_rmsnorm",
+    "zeda_compact_static", "zeda_moe_destroy", "zeda_last_error", "zeda_version",
 )
 
 
@@ -69,6 +70,8 @@ def _load() -> ctypes.CDLL:
     lib.zeda_moe_set_profiling.argtypes = [vp, i32]
     lib.zeda_moe_stage_ms.restype = i32
     lib.zeda_moe_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    lib.zeda_residual_rmsnorm.restype = i32
+    lib.zeda_residual_rmsnorm.argtypes = [vp, vp, vp, i32, i32, ctypes.c_float, vp]
     lib.zeda_compact_static.restype = i32
     lib.zeda_compact_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.zeda_moe_destroy.restype = i32
@@ -107,6 +110,20 @@ def workspace_bytes(cfg: Config) -> int:
 
 
 STATIC_MAX_TOKENS, STATIC_MAX_SLOTS = 4096, 32768
+
+
+def residual_rmsnorm(r: torch.Tensor, y: Optional[torch.Tensor], h: Optional[torch.Tensor] = None,
+                     eps: float = 1e-6) -> torch.Tensor:
+    """r <- bf16(r + y) in place (y may be None), returns h = RMSNorm(r) (gain-free) as bf16."""
+    assert r.is_cuda and r.dtype == torch.bfloat16 and r.dim() == 2 and r.is_contiguous()
+    if y is not None:
+        assert y.shape == r.shape and y.dtype == r.dtype and y.is_contiguous()
+    if h is None:
+        h = torch.empty_like(r)
+    with torch.cuda.device(r.device):
+        _check(lib.zeda_residual_rmsnorm(_ptr(r), _ptr(y), _ptr(h), r.shape[0], r.shape[1], float(eps),
+                                         _stream(r.device)))
+    return h
 
 
 def compact_static(topk_idx: torch.Tensor, n_real: int):

@@ -350,3 +350,55 @@ def test_pair_count_matches_flop_model():
     assert P == round(wl.T * wl.K * (1 - r))
     want = flops.moe_flops_zeda(wl.T, wl.d, wl.He, wl.E, wl.Z, wl.K, r)
     assert np.isclose(flops.expert_flops_pairs(P, wl.d, wl.He) + flops.router_flops(wl.T, wl.d, wl.E + wl.Z), want)
+
+
+# ---------------------------------------------------------------------------------- layer-stack glue
+
+def _bits(t):
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def test_residual_rmsnorm_closed_forms():
+    # a constant row c normalises to c / sqrt(c^2 + eps); the mean square of h is ms / (ms + eps)
+    import torch as _t
+    for c in (0.5, -2.0, 0.0):
+        r = _t.full((3, 128), c, dtype=_t.bfloat16)
+        nb, h = oracle.residual_rmsnorm(_bits(r), None, eps=1e-6)
+        assert np.array_equal(nb, _bits(r))
+        assert np.allclose(h, c / np.sqrt(c * c + 1e-6), rtol=0, atol=1e-15)
+    g = _t.Generator().manual_seed(3)
+    r = (_t.randn(7, 192, generator=g) * 4).to(_t.bfloat16)
+    _, h = oracle.residual_rmsnorm(_bits(r), None, eps=1e-6)
+    rd = r.double().numpy()
+    ms = (rd * rd).mean(axis=1)
+    assert np.allclose((h * h).mean(axis=1), ms / (ms + 1e-6), rtol=1e-13)
+    # scale invariance up to eps: normalising 8 r gives the same direction (power-of-two scale keeps bf16 exact)
+    _, h8 = oracle.residual_rmsnorm(_bits((r.float() * 8).to(_t.bfloat16)), None, eps=0.0)
+    _, h1 = oracle.residual_rmsnorm(_bits(r), None, eps=0.0)
+    assert np.allclose(h8, h1, rtol=1e-13)
+
+
+def test_residual_add_is_the_correctly_rounded_sum():
+    # brute force over bf16 operands against exact rational arithmetic: the stored residual is the
+    # bf16 nearest to r + y (ties to even), including pairs whose exponents are far apart
+    import fractions
+    import torch as _t
+    vals = _t.tensor([1.0, 1.0078125, -1.0078125, 3.0e-5, 255.0, 0.00390625, -0.0078125, 1.5, 6.1e-5, 128.5, 2.0 ** -20, 1.00390625],
+                     dtype=_t.float32).to(_t.bfloat16)
+    a = vals.repeat_interleave(len(vals)).view(1, -1)
+    b = vals.repeat(len(vals)).view(1, -1)
+    pad = 64 - a.shape[1] % 64
+    a = _t.cat([a, _t.zeros(1, pad, dtype=_t.bfloat16)], 1)
+    b = _t.cat([b, _t.zeros(1, pad, dtype=_t.bfloat16)], 1)
+    nb, _ = oracle.residual_rmsnorm(_bits(a), _bits(b))
+    got = (nb.astype(np.uint32) << 16).view(np.float32).astype(np.float64)[0]
+    for i in range(len(vals) ** 2):
+        exact = fractions.Fraction(float(a[0, i])) + fractions.Fraction(float(b[0, i]))
+        g = fractions.Fraction(float(got[i]))
+        if exact == 0:
+            assert g == 0
+            continue
+        # g is a bf16 value within half a bf16 ulp of the exact sum
+        e = np.floor(np.log2(abs(float(exact))))
+        ulp = fractions.Fraction(2) ** int(e - 7)
+        assert abs(g - exact) <= ulp / 2, (float(a[0, i]), float(b[0, i]), float(g))
