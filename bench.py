@@ -205,6 +205,123 @@ def time_forward(m, x, y, steps, warmup, flush, dist_barrier):
     return sum(per), per
 
 
+def run_stack(args, peaks, peaks_kind, dev, world, rank, barrier, dist):
+    """--workload stack: a pass through --layers stacked MoE blocks (attention excluded) with the
+    residual + RMSNorm glue between them.  One step = one pass of T tokens through every layer."""
+    from paper_2605_18643_b200 import zeda
+    layers, r0 = inputs.stack_layers(args.layers, T=args.stack_tokens)
+    T, d, He, E, Z, K = (layers[0].T, layers[0].d, layers[0].He, layers[0].E, layers[0].Z, layers[0].K)
+    mods = []
+    for l, wl in enumerate(layers):
+        wgu, wd = inputs.device_expert_weights(E, He, d, 100 + l, dev)
+        bias = None if wl.router_bias is None else wl.router_bias.to(dev)
+        mods.append(zeda.ZedaMoE(wl.router_w.to(dev), bias, wgu, wd, E, Z, K, T))
+    if rank > 0:
+        r0 = inputs.replica_tokens(layers[0], rank)
+    r_init = r0.to(dev)
+    r = r_init.clone()
+    h = torch.empty_like(r)
+    ys = [torch.empty_like(r), torch.empty_like(r)]
+
+    def one_pass():
+        r.copy_(r_init)
+        y = None
+        for l, m in enumerate(mods):
+            zeda.residual_rmsnorm(r, y, h)
+            y = m.forward(h, ys[l & 1])
+        return y
+
+    clocks = ClockSampler(dev.index or 0)
+    clocks.start()
+    for _ in range(args.warmup):
+        one_pass()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    barrier()
+    torch.cuda.synchronize()
+    for i in range(args.steps):
+        starts[i].record()
+        one_pass()
+        ends[i].record()
+    torch.cuda.synchronize()
+    barrier()
+    total_ms = sum(a.elapsed_time(b) for a, b in zip(starts, ends))
+    counters = [m.last_counters() for m in mods]
+    # stage events, one more pass
+    for m in mods:
+        m.set_profiling(True)
+    one_pass()
+    torch.cuda.synchronize()
+    stage = np.zeros(5)
+    for m in mods:
+        stage += np.array(m.stage_ms())
+        m.set_profiling(False)
+    # end to end: host residual in, host result out
+    r_pin = r0.pin_memory()
+    out_pin = torch.empty_like(r_pin).pin_memory()
+    e2e_s = 0.0
+    for i in range(args.warmup + args.steps):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        r_init.copy_(r_pin, non_blocking=True)
+        y = one_pass()
+        out_pin.copy_(y, non_blocking=True)
+        torch.cuda.synchronize()
+        if i >= args.warmup:
+            e2e_s += time.perf_counter() - t0
+    barrier()
+    clock_info = clocks.stop()
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_s = float(t[0]), float(t[1])
+    if rank == 0:
+        ms_per_step = total_ms / args.steps
+        hbm = peaks["hbm_gbs"] * 1e9
+        burst = peaks["bf16_tflops"]
+        sustained = peaks.get("bf16_tflops_sustained", burst)
+        t_roof = t_roof_s = 0.0
+        g1_bytes = g1_flops = 0
+        for (P, U, _, _) in counters:
+            t_roof += flops.layer_roofline_seconds(T, d, He, E + Z, P, U, burst * 1e12, hbm)[0]
+            t_roof_s += flops.layer_roofline_seconds(T, d, He, E + Z, P, U, sustained * 1e12, hbm)[0]
+            g1_bytes += U * 2 * He * d * 2 + T * d * 2 + P * He * 2
+            g1_flops += 4 * P * d * He
+        g1_s = stage[2] * 1e-3
+        if g1_bytes / hbm >= g1_flops / (sustained * 1e12):
+            roof = {"bound": "hbm", "achieved": g1_bytes / g1_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        else:
+            roof = {"bound": "tensor", "achieved": g1_flops / g1_s / 1e12, "peak": sustained, "unit": "TFLOP/s",
+                    "peak_kind": "sustained (kernel timed inside the step)", "peak_burst": burst}
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof.update(traffic=None, kernel="expert GEMM1 + SwiGLU, summed over the layers", peak_source=peaks_kind,
+                    algorithmic_bytes=g1_bytes, algorithmic_flops=g1_flops, kernel_ms=stage[2])
+        Ps = [c[0] for c in counters]
+        line = {
+            "metric": METRIC, "value": world * T / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "stack", "layers": len(mods), "T": T, "d": d, "d_expert": He, "n_real": E,
+                       "n_zero": Z, "top_k": K, "seed": 0, "pairs_per_layer_min_max": [min(Ps), max(Ps)],
+                       "zero_slot_fraction_mean": round(1.0 - sum(Ps) / (len(Ps) * T * K), 4),
+                       "weights_gb": round(len(mods) * E * 3 * d * He * 2 / 1e9, 2),
+                       "l2": "inputs larger than L2: every layer streams its own 1.2 GB of expert weights",
+                       "parallelism": "dp%d replicas, no collective" % world},
+            "clocks": clock_info,
+            "e2e": {"value": world * T * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": T * d * 2,
+                    "d2h_bytes_per_step": T * d * 2, "ms_per_step": 1e3 * e2e_s / args.steps},
+            "gpu_launches": (sum(c[3] for c in counters) + len(mods)) * args.steps,
+            "roofline": roof,
+            "layer_roofline": {"t_roof_us": t_roof * 1e6, "frac": t_roof / (ms_per_step * 1e-3),
+                               "t_roof_us_sustained": t_roof_s * 1e6,
+                               "frac_sustained": t_roof_s / (ms_per_step * 1e-3), "peak_source": peaks_kind},
+            "stage_ms": {n: float(v) for n, v in zip(["router", "sort", "gemm1", "gemm2", "combine"], stage)},
+        }
+        print(json.dumps(line))
+    for m in mods:
+        m.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -214,6 +331,8 @@ def main():
     ap.add_argument("--workload", default="decode")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-static", action="store_true")
+    ap.add_argument("--layers", type=int, default=48, help="layers of --workload stack")
+    ap.add_argument("--stack-tokens", type=int, default=4096, help="tokens per pass of --workload stack")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -239,6 +358,11 @@ def main():
     from paper_2605_18643_b200 import zeda  # raises if libzeda.so is missing
 
     peaks, peaks_kind = load_peaks()
+    if args.workload == "stack":
+        run_stack(args, peaks, peaks_kind, dev, world, rank, barrier, dist)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     wl = make_workload(args.workload)
     x_cpu = wl.x if rank == 0 else inputs.replica_tokens(wl, rank)
     m = zeda.from_workload(wl, dev)

@@ -18,38 +18,49 @@ __device__ __forceinline__ void fma_bf16x8(float (&acc)[8], float w, const uint4
     }
 }
 
-__global__ void __launch_bounds__(256)
+// One CTA per token, kCombineThreads threads, each owning every kCombineThreads-th 16-byte chunk of
+// the row (small CTAs: many tokens in flight per SM hide the dependent slot-table and row loads).
+constexpr int kCombineThreads = 64;
+
+__global__ void __launch_bounds__(kCombineThreads, 16)
 combine_kernel(const __nv_bfloat16 *__restrict__ obuf, const int32_t *__restrict__ inv,
                const float *__restrict__ topk_w, const __nv_bfloat16 *__restrict__ x, int K, int d,
                int copy_experts, __nv_bfloat16 *__restrict__ y) {
     pdl_launch_dependents();
     pdl_wait();
     const int t = blockIdx.x;
-    __shared__ int32_t s_pos[kMaxTopK];
-    __shared__ float s_w[kMaxTopK];
-    __shared__ float s_zero_mass;
-    if (threadIdx.x < K) {
-        s_pos[threadIdx.x] = inv[(size_t)t * K + threadIdx.x];
-        s_w[threadIdx.x] = topk_w[(size_t)t * K + threadIdx.x];
+    // every thread reads the token's slot table itself (K <= 16 entries, one cache line each way)
+    int32_t pos[kMaxTopK];
+    float w[kMaxTopK];
+    float zero_mass = 0.f;
+#pragma unroll
+    for (int k = 0; k < kMaxTopK; ++k) {
+        pos[k] = -1;
+        w[k] = 0.f;
+        if (k < K) {
+            pos[k] = __ldg(inv + (size_t)t * K + k);
+            w[k] = __ldg(topk_w + (size_t)t * K + k);
+            if (pos[k] < 0) zero_mass += w[k];
+        }
     }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float zm = 0.f;
-        for (int k = 0; k < K; ++k) if (s_pos[k] < 0) zm += s_w[k];
-        s_zero_mass = zm;
-    }
-    __syncthreads();
-    for (int c = blockIdx.y * blockDim.x + threadIdx.x; c < d / 8; c += gridDim.y * blockDim.x) {
+    for (int c = threadIdx.x; c < d / 8; c += kCombineThreads) {
         float acc[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-#pragma unroll 4
-        for (int k = 0; k < K; ++k) {
-            const int p = s_pos[k];
-            if (p >= 0) fma_bf16x8(acc, s_w[k], __ldg(reinterpret_cast<const uint4 *>(obuf + (size_t)p * d) + c));
+#pragma unroll
+        for (int k0 = 0; k0 < kMaxTopK; k0 += 8) {  // eight row loads are issued before the first use
+            if (k0 >= K) break;
+            uint4 v[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (k0 + k < K && pos[k0 + k] >= 0)
+                    v[k] = __ldg(reinterpret_cast<const uint4 *>(obuf + (size_t)pos[k0 + k] * d) + c);
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (k0 + k < K && pos[k0 + k] >= 0) fma_bf16x8(acc, w[k0 + k], v[k]);
         }
-        if (copy_experts && s_zero_mass != 0.f)
-            fma_bf16x8(acc, s_zero_mass, __ldg(reinterpret_cast<const uint4 *>(x + (size_t)t * d) + c));
+        if (copy_experts && zero_mass != 0.f)
+            fma_bf16x8(acc, zero_mass, __ldg(reinterpret_cast<const uint4 *>(x + (size_t)t * d) + c));
         uint4 o;
         uint32_t *ou = reinterpret_cast<uint32_t *>(&o);
 #pragma unroll
@@ -65,11 +76,7 @@ combine_kernel(const __nv_bfloat16 *__restrict__ obuf, const int32_t *__restrict
 
 int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s) {
     const zeda_moe_config_t &c = h->cfg;
-    // one 16-byte chunk per thread; small batches spread a row over several CTAs to fill the SMs
-    const int chunks = c.d_model / 8;
-    const int threads = (T >= 1024 && chunks >= 256) ? 256 : (T >= 256 && chunks >= 128 ? 128 : 64);
-    const int gy = (chunks + threads - 1) / threads;
-    const cudaError_t e = launch_kernel(h->pdl, combine_kernel, dim3(T, gy), dim3(threads), 0, s, h->ws.obuf, h->ws.inv,
+    const cudaError_t e = launch_kernel(h->pdl, combine_kernel, dim3(T), dim3(kCombineThreads), 0, s, h->ws.obuf, h->ws.inv,
                                         h->ws.topk_w, x, c.top_k, c.d_model, (int)(c.expert_kind == ZEDA_EXPERT_COPY), y);
     return e == cudaSuccess ? 1 : -1;
 }

@@ -464,19 +464,31 @@ slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n
     pdl_launch_dependents();
     pdl_wait();
     __shared__ ScanShared sh;
-    extern __shared__ int32_t pos[];       // [kPlaceWarps][n_real], then base[n_real]
+    extern __shared__ int32_t pos[];       // [kPlaceWarps][n_real], then base[n_real], then a histogram slab
     int32_t *base = pos + kPlaceWarps * n_real;
+    int32_t *slab = base + n_real;         // [kScanSlabInts]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int i = threadIdx.x; i < kPlaceWarps * n_real; i += blockDim.x) pos[i] = 0;
-    for (int e = threadIdx.x; e < n_real; e += blockDim.x) {
-        int before = 0, total = 0;
-        for (int b = 0; b < nblk; ++b) {
-            const int c = __ldg(block_hist + (size_t)b * n_real + e);
-            total += c;
-            if (b < (int)blockIdx.x) before += c;
+    for (int e = threadIdx.x; e < n_real; e += blockDim.x) { base[e] = 0; sh.cnt[e] = 0; }
+    // column sums of the CTA histograms: staged slab by slab with independent coalesced loads (a
+    // per-thread loop over global memory would be one L2 round trip after another)
+    const int slab_blocks = max(1, kScanSlabInts / n_real);
+    for (int b0 = 0; b0 < nblk; b0 += slab_blocks) {
+        const int nb = min(slab_blocks, nblk - b0);
+        const int32_t *g = block_hist + (size_t)b0 * n_real;
+        __syncthreads();
+        for (int i = threadIdx.x; i < nb * n_real; i += blockDim.x) slab[i] = __ldg(g + i);
+        __syncthreads();
+        for (int e = threadIdx.x; e < n_real; e += blockDim.x) {
+            int before = 0, total = 0;
+            for (int b = 0; b < nb; ++b) {
+                const int c = slab[b * n_real + e];
+                total += c;
+                if (b0 + b < (int)blockIdx.x) before += c;
+            }
+            base[e] += before;
+            sh.cnt[e] += total;
         }
-        base[e] = before;
-        sh.cnt[e] = total;
     }
     __syncthreads();
     finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, wl, blockIdx.x == 0);
@@ -659,7 +671,7 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
                       (const int32_t *)ws.topk_idx, T, K, c.n_real, ws.block_hist);
         if (nblk <= kFoldMaxBlocks) {
             launch_kernel(h->pdl, slot_scan_place_kernel, dim3(nblk), dim3(kPlaceWarps * 32),
-                          sizeof(int32_t) * (kPlaceWarps + 1) * c.n_real, s, (const int32_t *)ws.topk_idx, T, K, c.n_real,
+                          sizeof(int32_t) * ((kPlaceWarps + 1) * c.n_real + kScanSlabInts), s, (const int32_t *)ws.topk_idx, T, K, c.n_real,
                           nblk, (const int32_t *)ws.block_hist, ws.counts, ws.offsets, out.n_pairs, ws.meta, wl, ws.perm,
                           out.perm, ws.inv, ws.pair_token);
             launches = 3;

@@ -110,7 +110,7 @@ def _logits32(x: torch.Tensor, router_w: torch.Tensor, bias: Optional[torch.Tens
 def make_layer(name: str, T: int, d: int, He: int, E: int, Z: int, K: int, seed: int = 0,
                zero_fraction: Optional[float] = 0.5, zipf_s: float = 0.0,
                token_shift: float = 0.0, weight_seed: Optional[int] = None,
-               x: Optional[torch.Tensor] = None) -> Workload:
+               x: Optional[torch.Tensor] = None, with_experts: bool = True) -> Workload:
     """One layer's worth of seeded inputs.
 
     zero_fraction: target mean share of top-K slots on zero experts (ignored when Z == 0;
@@ -121,10 +121,12 @@ def make_layer(name: str, T: int, d: int, He: int, E: int, Z: int, K: int, seed:
         each token's zero logits move together by a * <x_t, u> ~ N(0, a^2) and the per-token
         zero share spreads from 0 to 100 %.
     x: optional caller-supplied activations (used by the layer stack); rows are never redrawn then.
+    with_experts: False leaves w_gate_up / w_down as None (the layer stack draws them on the device
+        with device_expert_weights: 58 GB of them do not pass through host memory).
     """
     assert K <= E + Z
     ws = seed if weight_seed is None else weight_seed
-    w_gate_up, w_down = expert_weights(E, He, d, ws)
+    w_gate_up, w_down = expert_weights(E, He, d, ws) if with_experts else (None, None)
     router_w = _normal((E + Z, d), 0.02, seed, _ID_ROUTER, torch.float32)
     own_x = x is None
     if own_x:
@@ -229,6 +231,34 @@ def static_reference(wl: Workload) -> Workload:
     bias = None if wl.router_bias is None else wl.router_bias[:wl.E].clone()
     return dataclasses.replace(wl, name=wl.name + "_static", Z=0, router_w=wl.router_w[:wl.E].clone(),
                                router_bias=bias, zero_bias=0.0, zero_fraction=0.0)
+
+
+def device_expert_weights(E: int, He: int, d: int, seed: int, device):
+    """Expert weights ~ N(0, 0.02^2) in bf16 drawn on `device` from a seeded generator of that
+    device (same shapes as expert_weights; a different, device-side random stream)."""
+    g = torch.Generator(device=device)
+    g.manual_seed(seed * 1000 + _ID_GATE_UP)
+    w_gate_up = torch.empty(E, 2 * He, d, dtype=torch.bfloat16, device=device)
+    w_down = torch.empty(E, d, He, dtype=torch.bfloat16, device=device)
+    for w in (w_gate_up, w_down):
+        for e in range(E):  # per expert: the fp32 scratch stays small
+            w[e] = (torch.randn(w[e].shape, generator=g, dtype=torch.float32, device=device) * 0.02).to(torch.bfloat16)
+    return w_gate_up, w_down
+
+
+def stack_layers(n_layers: int = 48, T: int = 4096, seed: int = 0, **over):
+    """Router-side inputs of a stack of Qwen3-30B-A3B-shaped MoE blocks (48 in the paper's models,
+    Section 4.2): per layer its own router rows and a zero-expert bias calibrated, on a proxy batch of
+    RMS-normalised N(0,1) tokens, to that layer's zero-slot target ~ U[0.3, 0.7].  Expert weights are
+    left out (see device_expert_weights).  Returns (list of Workloads, residual stream r0 [T, d])."""
+    kw = dict(QWEN)
+    kw.update(over)
+    fr = stack_layer_fractions(n_layers, seed)
+    proxy = rmsnorm_bf16(_normal((T, kw["d"]), 1.0, seed, _ID_X, torch.bfloat16, extra=77))
+    layers = [make_layer("stack_l%d" % l, T=T, seed=seed * 100 + l + 1, zero_fraction=fr[l], x=proxy,
+                         with_experts=False, **kw) for l in range(n_layers)]
+    r0 = _normal((T, kw["d"]), 1.0, seed, _ID_X, torch.bfloat16, extra=78)
+    return layers, r0
 
 
 def stack_layer_fractions(n_layers: int = 48, seed: int = 0):
