@@ -323,3 +323,20 @@ def test_routing_with_many_sort_blocks(zeda):
     l, idx, w, counts, offsets, perm, P = oracle_route(wl)
     check_route(m.route(wl.x.to(dev)), idx, w, counts, offsets, perm, P)
     m.close()
+
+
+# ---------------------------------------------------------------------------------- second model shape
+
+def test_glm_shaped_layer_and_net_point(zeda):
+    # Table of adapted models (Section 3.1): the second model has N=64, K=4, N_Z=32; its hidden
+    # sizes are not in the paper, so d and H_e are free parameters here.  NET (the paper's iso-FLOP
+    # static baseline) is the same layer with no zero experts and K/2 slots.
+    shape = dict(T=512, d=1024, He=512, E=64, Z=32, K=4)
+    wl = inputs.make_layer("glm_shaped", seed=12, zero_fraction=0.5, **shape)
+    err, (P, U, zs) = run_layer(zeda, wl, token_ids=sample_tokens(512, 40, 5))
+    assert abs(zs / (wl.T * wl.K) - 0.5) < 0.03
+    net = inputs.make_layer("glm_net", seed=12, zero_fraction=None, **dict(shape, Z=0, K=2))
+    err, (Pn, Un, zsn) = run_layer(zeda, net, token_ids=sample_tokens(512, 40, 6))
+    assert zsn == 0 and Pn == net.T * net.K
+    # NET spends K/2 expert evaluations per token; the zero-expert layer about K (1 - r_ZE) = K/2 on average
+    assert abs(P / Pn - 1.0) < 0.06
