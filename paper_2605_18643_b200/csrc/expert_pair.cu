@@ -196,7 +196,10 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA)
         if (leader && lane == 0) {
-            uint32_t it_count = 0, tile_count = 0;
+            uint32_t tile_count = 0;
+            uint32_t s = 0, ph = 0;  // ring stage of the next k-step and the parity of its use
+            // descriptors of stage 0; stage s is (s * kStageBytes) >> 4 further in the address field
+            const uint64_t a0 = smem_desc_sw128(ring), b0 = smem_desc_sw128(ring + kATileBytes);
             bool ok = true;
             for (long long item = first; item < n_items && ok; item += stride, ++tile_count) {
                 const Item it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
@@ -206,17 +209,16 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 if (!mbar_wait(bar_tempty + 8 * buf, tph ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d = tmem_base + buf * kAccCols;
-                for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
-                    const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
+                for (int ks = 0; ks < k_steps; ++ks) {
                     if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = ring + s * kStageBytes;
-                    const uint64_t a = smem_desc_sw128(sa);
-                    const uint64_t b = smem_desc_sw128(sa + kATileBytes);
+                    const uint64_t a = a0 + (uint64_t)(s * (kStageBytes >> 4));
+                    const uint64_t b = b0 + (uint64_t)(s * (kStageBytes >> 4));
 #pragma unroll
                     for (int k = 0; k < kBlockK / 16; ++k)  // +32 bytes per 16-element k slice inside the swizzle row
                         umma_bf16_pair(d, a + 2 * k, b + 2 * k, idesc, (ks | k) ? 1u : 0u);
                     umma_commit_pair(bar_empty + 8 * s);  // the stage is free in both CTAs once these MMAs have read it
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
                 umma_commit_pair(bar_tfull + 8 * buf);    // accumulators complete in both CTAs
