@@ -203,6 +203,17 @@ zeda_status_t zeda_compact_static(const int32_t *topk_idx, int32_t T, int32_t to
                                   int32_t *expert_counts, int32_t *expert_offsets, int32_t *perm,
                                   int32_t *n_pairs, void *stream);
 
+/* Failure reporting.  Every device-side wait in the tensor-core kernels is bounded; a wait that
+ * expires makes its CTA record an error word in the workspace, skip its remaining work and leave
+ * normally (the context stays usable, the call's outputs are undefined).  The word is sticky:
+ * zeda_moe_last_counters and zeda_moe_destroy report ZEDA_ERR_TIMEOUT until it is cleared.
+ *   zeda_moe_selftest_wait  exercises that path without a fault: a one-thread kernel waits, for at
+ *                           most limit_us microseconds (1..100000), on a barrier that nothing signals,
+ *                           and records the expiry like the kernels do.  Asynchronous on the stream.
+ *   zeda_moe_clear_error    resets the error word (stream-ordered). */
+zeda_status_t zeda_moe_selftest_wait(zeda_moe_t *h, int32_t limit_us, void *stream);
+zeda_status_t zeda_moe_clear_error(zeda_moe_t *h, void *stream);
+
 /* Reports a pending device-side error word (ZEDA_ERR_TIMEOUT) if any, then releases the handle.
  * Does not touch caller-owned device memory. */
 zeda_status_t zeda_moe_destroy(zeda_moe_t *h);

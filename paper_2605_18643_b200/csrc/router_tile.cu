@@ -169,7 +169,25 @@ router_logits_tile_kernel(const __grid_constant__ CUtensorMap map_w, const __gri
 
 constexpr int kSmemBytes = kStages * kStageBytes + 1024;
 
+// Self-test of the bounded wait: one thread waits on an mbarrier that nothing will ever arrive on,
+// with a short limit, and records the expiry in the handle's error word exactly as the kernels do.
+__global__ void wait_selftest_kernel(int32_t *__restrict__ meta, long long limit_cycles) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!mbar_wait_for(smem_u32(&bar), 0, &s_abort, limit_cycles)) atomicExch(&meta[kMetaError], 99);
+    }
+}
+
 }  // namespace
+
+int launch_wait_selftest(const zeda_moe *h, long long limit_cycles, cudaStream_t s) {
+    wait_selftest_kernel<<<1, 32, 0, s>>>(h->ws.meta, limit_cycles);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
 
 int router_split_pad(int n_cand) { return (n_cand + 127) / 128 * 128; }
 

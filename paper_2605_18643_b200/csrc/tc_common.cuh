@@ -39,7 +39,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // Bounded wait: false if the limit passed or another role already gave up.  The common case (the
 // phase completes within a few thousand polls) reads no timer at all; after that the SM's own
 // cycle counter bounds the wait.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool mbar_wait_for(uint32_t bar, uint32_t parity, volatile int *abort_flag, long long limit_cycles) {
 #pragma unroll 1
     for (int i = 0; i < 4096; ++i)
         if (mbar_try(bar, parity)) return true;
@@ -48,10 +48,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     while (!mbar_try(bar, parity)) {
         if ((++spins & 255) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) return false;
+            if (clock64() - t0 > limit_cycles) return false;
         }
     }
     return true;
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    return mbar_wait_for(bar, parity, abort_flag, kWaitLimitCycles);
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2, uint32_t bar) {

@@ -326,6 +326,29 @@ zeda_status_t zeda_moe_last_counters(zeda_moe_t *h, int64_t out[4], void *stream
     return ZEDA_OK;
 }
 
+zeda_status_t zeda_moe_selftest_wait(zeda_moe_t *h, int32_t limit_us, void *stream) {
+    if (!h) { set_error("handle is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    if (limit_us < 1 || limit_us > 100000) { set_error("limit_us must be in [1, 100000]"); return ZEDA_ERR_INVALID_ARG; }
+    cudaError_t e = cudaSetDevice(h->cfg.device);
+    if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
+    int khz = 0;
+    e = cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, h->cfg.device);
+    if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute", e);
+    const long long cycles = (long long)limit_us * (khz > 0 ? khz : 1000000) / 1000;
+    if (launch_wait_selftest(h, cycles, static_cast<cudaStream_t>(stream)) < 0)
+        return cuda_fail("self-test launch", cudaGetLastError());
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_moe_clear_error(zeda_moe_t *h, void *stream) {
+    if (!h) { set_error("handle is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    cudaError_t e = cudaSetDevice(h->cfg.device);
+    if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
+    e = cudaMemsetAsync(h->ws.meta + kMetaError, 0, sizeof(int32_t), static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
+    return ZEDA_OK;
+}
+
 zeda_status_t zeda_moe_set_profiling(zeda_moe_t *h, int32_t enable) {
     if (!h) { set_error("handle is NULL"); return ZEDA_ERR_INVALID_ARG; }
     cudaError_t e = cudaSetDevice(h->cfg.device);

@@ -112,6 +112,7 @@ int launch_experts_gemm2_tile(const zeda_moe *h, int T, cudaStream_t s);
 int init_pair_kernels(zeda_moe *h);
 int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
 int launch_experts_gemm2_pair(const zeda_moe *h, int T, cudaStream_t s);
+int launch_wait_selftest(const zeda_moe *h, long long limit_cycles, cudaStream_t s);
 int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s);
 
 void set_error(const char *fmt, ...);

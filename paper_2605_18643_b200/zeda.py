@@ -25,6 +25,7 @@ EXPORTS = (
     "zeda_moe_workspace_bytes", "zeda_moe_create", "zeda_route", "zeda_route_from_logits",
     "zeda_router_logits", "zeda_moe_forward", "zeda_moe_forward_host", "zeda_moe_stats",
     "zeda_moe_last_counters", "zeda_moe_set_profiling", "zeda_moe_stage_ms", "zeda_residual_rmsnorm",
+    "zeda_moe_selftest_wait", "zeda_moe_clear_error",
     "zeda_compact_static", "zeda_moe_destroy", "zeda_last_error", "zeda_version",
 )
 
@@ -70,6 +71,10 @@ def _load() -> ctypes.CDLL:
     lib.zeda_moe_set_profiling.argtypes = [vp, i32]
     lib.zeda_moe_stage_ms.restype = i32
     lib.zeda_moe_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    lib.zeda_moe_selftest_wait.restype = i32
+    lib.zeda_moe_selftest_wait.argtypes = [vp, i32, vp]
+    lib.zeda_moe_clear_error.restype = i32
+    lib.zeda_moe_clear_error.argtypes = [vp, vp]
     lib.zeda_residual_rmsnorm.restype = i32
     lib.zeda_residual_rmsnorm.argtypes = [vp, vp, vp, i32, i32, ctypes.c_float, vp]
     lib.zeda_compact_static.restype = i32
@@ -243,6 +248,13 @@ class ZedaMoE:
         out = (ctypes.c_int64 * 4)()
         _check(lib.zeda_moe_last_counters(self._h, out, _stream(self.device)))
         return tuple(int(v) for v in out)
+
+    def selftest_wait(self, limit_us: int = 1000):
+        """Makes a bounded device wait expire on purpose (no fault): the next last_counters() raises."""
+        _check(lib.zeda_moe_selftest_wait(self._h, int(limit_us), _stream(self.device)))
+
+    def clear_error(self):
+        _check(lib.zeda_moe_clear_error(self._h, _stream(self.device)))
 
     def set_profiling(self, enable: bool):
         _check(lib.zeda_moe_set_profiling(self._h, 1 if enable else 0))

@@ -340,3 +340,25 @@ def test_glm_shaped_layer_and_net_point(zeda):
     assert zsn == 0 and Pn == net.T * net.K
     # NET spends K/2 expert evaluations per token; the zero-expert layer about K (1 - r_ZE) = K/2 on average
     assert abs(P / Pn - 1.0) < 0.06
+
+
+def test_expired_device_wait_is_reported_and_the_handle_stays_usable(zeda):
+    # failure detection without a fault: a wait with a 1 ms limit on a barrier that nothing signals
+    wl = inputs.tiny(seed=9)
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev)
+    x = wl.x.to(dev)
+    y0 = m.forward(x).view(torch.int16).clone()
+    m.last_counters()                       # no error pending
+    m.selftest_wait(limit_us=1000)
+    with pytest.raises(zeda.ZedaError) as e:
+        m.last_counters()
+    assert e.value.status == -5 and "wait expired" in str(e.value)
+    with pytest.raises(zeda.ZedaError):     # sticky until cleared
+        m.last_counters()
+    m.clear_error()
+    y1 = m.forward(x).view(torch.int16)
+    torch.cuda.synchronize()
+    assert torch.equal(y0, y1)
+    m.last_counters()
+    m.close()
