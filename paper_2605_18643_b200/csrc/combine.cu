@@ -43,7 +43,7 @@ combine_kernel(const __nv_bfloat16 *__restrict__ obuf, const int32_t *__restrict
             if (pos[k] < 0) zero_mass += w[k];
         }
     }
-    for (int c = threadIdx.x; c < d / 8; c += kCombineThreads) {
+    for (int c = blockIdx.y * kCombineThreads + threadIdx.x; c < d / 8; c += gridDim.y * kCombineThreads) {
         float acc[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc[i] = 0.f;
@@ -76,7 +76,11 @@ combine_kernel(const __nv_bfloat16 *__restrict__ obuf, const int32_t *__restrict
 
 int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s) {
     const zeda_moe_config_t &c = h->cfg;
-    const cudaError_t e = launch_kernel(h->pdl, combine_kernel, dim3(T), dim3(kCombineThreads), 0, s, h->ws.obuf, h->ws.inv,
+    // small batches spread a row over several CTAs so that the grid still covers the SMs
+    const int chunks = c.d_model / 8;
+    int gy = 1;
+    while (T * gy < 4 * h->sm_count && gy * kCombineThreads < chunks) gy *= 2;
+    const cudaError_t e = launch_kernel(h->pdl, combine_kernel, dim3(T, gy), dim3(kCombineThreads), 0, s, h->ws.obuf, h->ws.inv,
                                         h->ws.topk_w, x, c.top_k, c.d_model, (int)(c.expert_kind == ZEDA_EXPERT_COPY), y);
     return e == cudaSuccess ? 1 : -1;
 }

@@ -23,6 +23,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 // per candidate row, lanes striding the feature axis with 16-byte loads.
 // ---------------------------------------------------------------------------------------------
 constexpr int kTok = 8;
+constexpr int kRouterUnroll = 8;  // 16-byte weight loads a lane keeps in flight
 
 __global__ void __launch_bounds__(256)
 router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restrict__ router_w,
@@ -50,13 +51,13 @@ router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restric
 #pragma unroll
         for (int r = 0; r < kTok; ++r) acc[r] = 0.f;
         const float4 *wrow = reinterpret_cast<const float4 *>(router_w + (size_t)j * d);
-        for (int c4 = lane; c4 < d / 4; c4 += 128) {
-            float4 w[4];
+        for (int c4 = lane; c4 < d / 4; c4 += 32 * kRouterUnroll) {
+            float4 w[kRouterUnroll];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)  // four independent 16-byte loads in flight per lane
+            for (int u = 0; u < kRouterUnroll; ++u)  // independent 16-byte loads in flight per lane
                 w[u] = (c4 + 32 * u < d / 4) ? __ldg(wrow + c4 + 32 * u) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < kRouterUnroll; ++u) {
                 if (c4 + 32 * u < d / 4) {
 #pragma unroll
                     for (int r = 0; r < kTok; ++r) {
