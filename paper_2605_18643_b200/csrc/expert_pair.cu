@@ -141,8 +141,11 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         if (lane == 0) {
             uint32_t it_count = 0;
             bool ok = true;
+            Item nxt = {0, 0, 0, 0};  // the next item's description is fetched while this one is processed
+            if (first < n_items) nxt = load_item(first, m_blocks, tile_expert, tile_row0, counts, offsets);
             for (long long item = first; item < n_items && ok; item += stride) {
-                const Item it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
+                const Item it = nxt;
+                if (item + stride < n_items) nxt = load_item(item + stride, m_blocks, tile_expert, tile_row0, counts, offsets);
                 const int half = ((it.n + 31) >> 5) << 4;  // B rows of this CTA; the tile has 2 * half columns
                 const uint32_t bytes = 2u * (uint32_t)(kATileBytes + (MODE == 2 ? half * kRowBytes : 0));
                 for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
@@ -168,8 +171,11 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         if (lane == 0) {
             uint32_t it_count = 0;
             bool ok = true;
+            Item nxt = {0, 0, 0, 0};  // the next item's description is fetched while this one is processed
+            if (first < n_items) nxt = load_item(first, m_blocks, tile_expert, tile_row0, counts, offsets);
             for (long long item = first; item < n_items && ok; item += stride) {
-                const Item it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
+                const Item it = nxt;
+                if (item + stride < n_items) nxt = load_item(item + stride, m_blocks, tile_expert, tile_row0, counts, offsets);
                 const int half = ((it.n + 31) >> 5) << 4;
                 const int brow0 = (int)rank * half;  // first tile column / pair row this CTA loads
                 for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
@@ -201,8 +207,11 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             // descriptors of stage 0; stage s is (s * kStageBytes) >> 4 further in the address field
             const uint64_t a0 = smem_desc_sw128(ring), b0 = smem_desc_sw128(ring + kATileBytes);
             bool ok = true;
+            Item nxt = {0, 0, 0, 0};  // the next item's description is fetched while this one is processed
+            if (first < n_items) nxt = load_item(first, m_blocks, tile_expert, tile_row0, counts, offsets);
             for (long long item = first; item < n_items && ok; item += stride, ++tile_count) {
-                const Item it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
+                const Item it = nxt;
+                if (item + stride < n_items) nxt = load_item(item + stride, m_blocks, tile_expert, tile_row0, counts, offsets);
                 const int n_cols = ((it.n + 31) >> 5) << 5;
                 const uint32_t idesc = instr_desc_pair(n_cols);
                 const uint32_t buf = tile_count & 1u, tph = (tile_count >> 1) & 1u;
@@ -258,8 +267,11 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         const uint32_t dst_off = (uint32_t)(rsub * kRowBytes + ((chunk ^ (rsub & 7)) << 4));
         uint32_t it_count = 0;
         bool ok = true;
+        Item nxt = {0, 0, 0, 0};  // the next item's description is fetched while this one is processed
+        if (first < n_items) nxt = load_item(first, m_blocks, tile_expert, tile_row0, counts, offsets);
         for (long long item = first; item < n_items && ok; item += stride) {
-            const Item it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
+            const Item it = nxt;
+            if (item + stride < n_items) nxt = load_item(item + stride, m_blocks, tile_expert, tile_row0, counts, offsets);
             const int half = ((it.n + 31) >> 5) << 4;
             const int brow0 = (int)rank * half;
             const __nv_bfloat16 *src[HALF_MAX / 16];
@@ -296,8 +308,11 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         const int prow = lane >> 2, pch = lane & 3;  // 16-byte piece this lane stores: rows prow + 8 i, features 8 pch ..
         uint32_t tile_count = 0;
         bool ok = true;
+        Item nxt = {0, 0, 0, 0};  // the next item's description is fetched while this one is processed
+        if (first < n_items) nxt = load_item(first, m_blocks, tile_expert, tile_row0, counts, offsets);
         for (long long item = first; item < n_items && ok; item += stride, ++tile_count) {
-            const Item it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
+            const Item it = nxt;
+            if (item + stride < n_items) nxt = load_item(item + stride, m_blocks, tile_expert, tile_row0, counts, offsets);
             const uint32_t buf = tile_count & 1u, tph = (tile_count >> 1) & 1u;
             ok = mbar_wait(bar_tfull + 8 * buf, tph, abort_flag);
             ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp before the aligned TMEM loads
