@@ -18,6 +18,9 @@
  *   - Calls enqueue work on the given cudaStream_t (passed as void*, NULL = default stream) and
  *     return without synchronising, except where stated.  Outputs are valid once the stream has
  *     been synchronised.  A handle is not thread-safe; distinct handles are independent.
+ *   - zeda_moe_forward, zeda_route and zeda_residual_rmsnorm only enqueue kernels and device-to-device
+ *     copies: a call can be captured in a CUDA graph and replayed on new contents of the same buffers
+ *     (the buffer addresses and T are part of the captured launches).
  *   - Every entry point returns a zeda_status_t (ZEDA_OK = 0); nothing throws, aborts or traps.
  *     Arguments are checked before anything is launched; zeda_last_error() gives a text for the
  *     last failure on the calling thread.

@@ -362,3 +362,33 @@ def test_expired_device_wait_is_reported_and_the_handle_stays_usable(zeda):
     assert torch.equal(y0, y1)
     m.last_counters()
     m.close()
+
+
+def test_forward_can_be_captured_in_a_cuda_graph(zeda):
+    # the call enqueues kernels only (no allocation, no host synchronisation): it can be captured once
+    # and replayed on new contents of the same buffers
+    wl = inputs.tiny(seed=13, T=300)
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev)
+    x = wl.x.to(dev)
+    y = torch.empty_like(x)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for _ in range(2):
+            m.forward(x, y)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            m.forward(x, y)
+    torch.cuda.synchronize()
+    x2 = inputs.tiny(seed=14, T=300).x.to(dev)
+    for src in (x2, wl.x.to(dev)):
+        x.copy_(src)
+        graph.replay()
+        torch.cuda.synchronize()
+        got = y.view(torch.int16).clone()
+        want = m.forward(src.clone()).view(torch.int16)
+        torch.cuda.synchronize()
+        assert torch.equal(got, want)
+    del graph
+    m.close()
