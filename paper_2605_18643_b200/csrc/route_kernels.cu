@@ -90,14 +90,23 @@ constexpr int kRegsPerLane = kMaxCand / 32;
 
 // Top-K and routing weights of one token by one warp.  On return lane k < K holds slot k.
 // RPL = logits per lane (32 * RPL >= n_cand).
+// The row may arrive as n_parts partial sums, part_stride floats apart; they are added in order.
 template <int RPL>
-__device__ __forceinline__ void topk_gate_token(const float *__restrict__ row, int n_real, int n_cand, int K,
+__device__ __forceinline__ void topk_gate_token(const float *__restrict__ row, int n_parts, size_t part_stride,
+                                                int n_real, int n_cand, int K,
                                                 int gate_mode, int lane, int &my_idx, float &my_w) {
     float v[RPL];
 #pragma unroll
     for (int r = 0; r < RPL; ++r) {
         const int j = r * 32 + lane;
         v[r] = (j < n_cand) ? row[j] : -INFINITY;
+    }
+    for (int p = 1; p < n_parts; ++p) {
+#pragma unroll
+        for (int r = 0; r < RPL; ++r) {
+            const int j = r * 32 + lane;
+            if (j < n_cand) v[r] += row[p * part_stride + j];
+        }
     }
     // row maximum and softmax denominator over all candidates
     float m = v[0];
@@ -150,7 +159,7 @@ __device__ __forceinline__ void topk_gate_token(const float *__restrict__ row, i
 
 template <int RPL>
 __global__ void __launch_bounds__(256)
-topk_gate_kernel(const float *__restrict__ logits, int T, int n_real, int n_cand, int K, int gate_mode,
+topk_gate_kernel(const float *__restrict__ logits, int n_parts, int T, int n_real, int n_cand, int K, int gate_mode,
                  int32_t *__restrict__ topk_idx, float *__restrict__ topk_w) {
     pdl_launch_dependents();
     pdl_wait();
@@ -159,7 +168,8 @@ topk_gate_kernel(const float *__restrict__ logits, int T, int n_real, int n_cand
     if (t >= T) return;
     int my_idx;
     float my_w;
-    topk_gate_token<RPL>(logits + (size_t)t * n_cand, n_real, n_cand, K, gate_mode, lane, my_idx, my_w);
+    topk_gate_token<RPL>(logits + (size_t)t * n_cand, n_parts, (size_t)T * n_cand, n_real, n_cand, K, gate_mode, lane,
+                         my_idx, my_w);
     if (lane < K) {
         topk_idx[(size_t)t * K + lane] = my_idx;
         topk_w[(size_t)t * K + lane] = my_w;
@@ -353,7 +363,7 @@ route_small_kernel(const float *__restrict__ logits, int T, int n_real, int n_ca
     if (t < T) {
         int my_idx;
         float my_w;
-        topk_gate_token<RPL>(logits + (size_t)t * n_cand, n_real, n_cand, K, gate_mode, lane, my_idx, my_w);
+        topk_gate_token<RPL>(logits + (size_t)t * n_cand, 1, 0, n_real, n_cand, K, gate_mode, lane, my_idx, my_w);
         if (lane < K) {
             topk_idx[(size_t)t * K + lane] = my_idx;
             topk_w[(size_t)t * K + lane] = my_w;
@@ -623,9 +633,14 @@ int init_route_kernels(const zeda_moe *h) {
     return 0;
 }
 
-int launch_router_logits(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, cudaStream_t s) {
+int launch_router_logits(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, cudaStream_t s, int *n_parts) {
+    if (n_parts) *n_parts = 1;
     // large batches: the GEMM goes to the tensor cores (exact three-way bf16 split of the weights)
-    if (T >= 256 && h->router_maps) return launch_router_logits_tile(h, x, T, logits, s);
+    if (T >= 256 && h->router_maps) {
+        const int split = n_parts ? router_split_factor(h, T) : 1;
+        if (n_parts) *n_parts = split;
+        return launch_router_logits_tile(h, x, T, logits, split, s);
+    }
     const int d = h->cfg.d_model, n_cand = h->cfg.n_real + h->cfg.n_zero;
     const int tiles = (T + kTok - 1) / kTok;
     // split the candidates over grid.y until the grid covers the SMs about twice
@@ -640,7 +655,7 @@ int launch_router_logits(const zeda_moe *h, const __nv_bfloat16 *x, int T, float
     return e == cudaSuccess ? 1 : -1;
 }
 
-int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, const RouteOut &out, cudaStream_t s) {
+int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, const RouteOut &out, cudaStream_t s, int n_parts) {
     const zeda_moe_config_t &c = h->cfg;
     const int n_cand = c.n_real + c.n_zero, K = c.top_k;
     const Workspace &ws = h->ws;
@@ -664,7 +679,7 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
         launches = 1;
     } else {
 #define ZEDA_CALL_TOPK(R) \
-    launch_kernel(h->pdl, topk_gate_kernel<R>, dim3((T + 7) / 8), dim3(256), 0, s, logits, T, c.n_real, n_cand, K, \
+    launch_kernel(h->pdl, topk_gate_kernel<R>, dim3((T + 7) / 8), dim3(256), 0, s, logits, n_parts, T, c.n_real, n_cand, K, \
                   c.gate_mode, ws.topk_idx, ws.topk_w)
         ZEDA_RPL_DISPATCH(ZEDA_CALL_TOPK);
 #undef ZEDA_CALL_TOPK

@@ -46,7 +46,7 @@ split_router_kernel(const float *__restrict__ w, int n_cand, int nc_pad, int d, 
 
 __global__ void __launch_bounds__(kThreads, 1)
 router_logits_tile_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x,
-                          const float *__restrict__ bias, int T, int n_cand, int m_tiles, int k_steps,
+                          const float *__restrict__ bias, int T, int n_cand, int m_tiles, int k_steps, int split,
                           int32_t *__restrict__ meta, float *__restrict__ logits) {
     pdl_launch_dependents();
     extern __shared__ __align__(1024) unsigned char router_smem[];
@@ -74,23 +74,28 @@ router_logits_tile_kernel(const __grid_constant__ CUtensorMap map_w, const __gri
     const uint32_t tmem_base = s_tmem_base;
     volatile int *abort_flag = &s_abort;
     pdl_wait();
+    // Work item = (token tile, candidate tile, slice of the reduction axis).  With few token tiles the
+    // reduction axis is cut into `split` slices so that the grid still covers the SMs; slice p writes
+    // its partial sums to logits + p * T * n_cand and the top-K kernel adds the slices in order.
     const int tok_tiles = (T + kTokTile - 1) / kTokTile;
-    const int n_items = tok_tiles * m_tiles;
+    const int n_items = tok_tiles * m_tiles * split;
+    k_steps /= split;  // per item
 
     if (warp == 0) {
         if (lane == 0) {
             uint32_t it_count = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-                const int mt = item % m_tiles, tt = item / m_tiles;
+                const int sp = item % split, mt = (item / split) % m_tiles, tt = item / (split * m_tiles);
                 for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
                     const uint32_t s = it_count % kStages, ph = (it_count / kStages) & 1u;
                     if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t full = bar_full + 8 * s, sa = ring + s * kStageBytes;
+                    const int kc = (sp * k_steps + ks) * kBlockK;
                     mbar_expect_tx(full, kStageBytes);
                     for (int piece = 0; piece < 3; ++piece)
-                        tma_load_3d(sa + piece * kTileBytes, &map_w, ks * kBlockK, mt * 128, piece, full);
-                    tma_load_2d(sa + 3 * kTileBytes, &map_x, ks * kBlockK, tt * kTokTile, full);
+                        tma_load_3d(sa + piece * kTileBytes, &map_w, kc, mt * 128, piece, full);
+                    tma_load_2d(sa + 3 * kTileBytes, &map_x, kc, tt * kTokTile, full);
                 }
             }
             if (!ok) { if (!*abort_flag) atomicExch(&meta[kMetaError], 4); s_abort = 1; }
@@ -130,13 +135,14 @@ router_logits_tile_kernel(const __grid_constant__ CUtensorMap map_w, const __gri
         uint32_t tile_count = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++tile_count) {
-            const int mt = item % m_tiles, tt = item / m_tiles;
+            const int sp = item % split, mt = (item / split) % m_tiles, tt = item / (split * m_tiles);
             if (!mbar_wait(bar_tfull, tile_count & 1u, abort_flag)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
             const int j = mt * 128 + 32 * q + lane;  // candidate of this lane
-            const float b = (bias && j < n_cand) ? __ldg(bias + j) : 0.f;
+            const float b = (bias && j < n_cand && sp == 0) ? __ldg(bias + j) : 0.f;  // slice 0 carries the bias
+            float *out = logits + (size_t)sp * T * n_cand;
             const uint32_t t0 = tmem_base + ((uint32_t)(32 * q) << 16);
             const int tok0 = tt * kTokTile;
             for (int c0 = 0; c0 < kTokTile; c0 += 32) {
@@ -153,7 +159,7 @@ router_logits_tile_kernel(const __grid_constant__ CUtensorMap map_w, const __gri
 #pragma unroll
                     for (int c = 0; c < 32; ++c)
                         if (tok0 + c0 + c < T)
-                            logits[(size_t)(tok0 + c0 + c) * n_cand + j] = ((lo[c] + mid[c]) + hi[c]) + b;
+                            out[(size_t)(tok0 + c0 + c) * n_cand + j] = ((lo[c] + mid[c]) + hi[c]) + b;
                 }
             }
         }
@@ -208,7 +214,18 @@ int init_router_tile(zeda_moe *h) {
     return 0;
 }
 
-int launch_router_logits_tile(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, cudaStream_t s) {
+int router_split_factor(const zeda_moe *h, int T) {
+    const int nc_pad = router_split_pad(h->cfg.n_real + h->cfg.n_zero);
+    const int items = (T + kTokTile - 1) / kTokTile * (nc_pad / 128);
+    const int k_steps = h->cfg.d_model / kBlockK;
+    int split = 1;
+    while (split < kRouterMaxSplit && items * split * 2 <= h->sm_count && k_steps % (split * 2) == 0 &&
+           (long long)T * split * 2 <= router_part_rows(h->cfg.max_tokens))
+        split *= 2;
+    return split;
+}
+
+int launch_router_logits_tile(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, int split, cudaStream_t s) {
     const zeda_moe_config_t &c = h->cfg;
     const int n_cand = c.n_real + c.n_zero, nc_pad = router_split_pad(n_cand);
     // the activations are the caller's buffer of this call: their tensor map is made per call (host only)
@@ -219,11 +236,11 @@ int launch_router_logits_tile(const zeda_moe *h, const __nv_bfloat16 *x, int T, 
     if (!encode_bf16_map(&map_x, x, 2, dims, strides, box)) return -1;
     const RouterMaps *rm = static_cast<const RouterMaps *>(h->router_maps);
     const int m_tiles = nc_pad / 128;
-    const int n_items = (T + kTokTile - 1) / kTokTile * m_tiles;
+    const int n_items = (T + kTokTile - 1) / kTokTile * m_tiles * split;
     const int grid = n_items < h->sm_count ? n_items : h->sm_count;
     const cudaError_t e = launch_kernel(h->pdl, router_logits_tile_kernel, dim3(grid), dim3(kThreads), kSmemBytes, s,
                                         rm->w_split, map_x, h->router_bias, T, n_cand, m_tiles, c.d_model / kBlockK,
-                                        h->ws.meta, logits);
+                                        split, h->ws.meta, logits);
     return e == cudaSuccess ? 1 : -1;
 }
 

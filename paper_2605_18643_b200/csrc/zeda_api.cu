@@ -71,7 +71,7 @@ size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int
     w.tile_row0 = (int32_t *)take(tiles * 4);
     w.ptile_expert = (int32_t *)take(tiles * 4);
     w.ptile_row0 = (int32_t *)take(tiles * 4);
-    w.logits = (float *)take((size_t)c.max_tokens * n_cand * 4);
+    w.logits = (float *)take((size_t)router_part_rows(c.max_tokens) * n_cand * 4);
     w.stat_part = (float *)take(nblk_stats * 2 * n_cand * 4);
     // pair buffers carry one tile of slack rows so that a full tile may be read past the last pair
     w.hmid = (__nv_bfloat16 *)take((slots + kPairTileM) * c.d_expert * 2);
@@ -104,16 +104,18 @@ zeda_status_t check_call(zeda_moe_t *h, const void *in, int32_t T, const char *i
 }
 
 // Routing into the workspace (+ optional user copies); returns launches or <0.
-int route_into(zeda_moe_t *h, const __nv_bfloat16 *x, const float *logits_in, int T, const RouteOut &out, cudaStream_t s) {
-    int n = 0;
+// full_logits: the caller reads ws.logits afterwards, so the router may not leave them in slices.
+int route_into(zeda_moe_t *h, const __nv_bfloat16 *x, const float *logits_in, int T, const RouteOut &out, cudaStream_t s,
+               bool full_logits = false) {
+    int n = 0, n_parts = 1;
     const float *logits = logits_in;
     if (!logits) {
-        int r = launch_router_logits(h, x, T, h->ws.logits, s);
+        int r = launch_router_logits(h, x, T, h->ws.logits, s, full_logits ? nullptr : &n_parts);
         if (r < 0) return r;
         n += r;
         logits = h->ws.logits;
     }
-    int r = launch_route_from_logits(h, logits, T, out, s);
+    int r = launch_route_from_logits(h, logits, T, out, s, n_parts);
     if (r < 0) return r;
     return n + r;
 }
@@ -122,11 +124,12 @@ zeda_status_t forward_device(zeda_moe_t *h, const __nv_bfloat16 *x, int T, __nv_
     const bool prof = h->profiling;
     auto mark = [&](int i) { if (prof) cudaEventRecord(h->ev[i], s); };
     mark(0);
-    int n = launch_router_logits(h, x, T, h->ws.logits, s);
+    int n_parts = 1;
+    int n = launch_router_logits(h, x, T, h->ws.logits, s, &n_parts);
     if (n < 0) return cuda_fail("router launch", cudaGetLastError());
     mark(1);
     RouteOut none = {};
-    int r = launch_route_from_logits(h, h->ws.logits, T, none, s);
+    int r = launch_route_from_logits(h, h->ws.logits, T, none, s, n_parts);
     if (r < 0) return cuda_fail("routing launch", cudaGetLastError());
     n += r;
     mark(2);
@@ -300,7 +303,7 @@ zeda_status_t zeda_moe_stats(zeda_moe_t *h, const void *x, int32_t T, float *f, 
     if (st != ZEDA_OK || T == 0) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     RouteOut none = {};
-    int n = route_into(h, static_cast<const __nv_bfloat16 *>(x), nullptr, T, none, s);
+    int n = route_into(h, static_cast<const __nv_bfloat16 *>(x), nullptr, T, none, s, true);
     if (n < 0) return cuda_fail("routing launch", cudaGetLastError());
     int r = launch_stats(h, h->ws.logits, h->ws.topk_idx, T, f, p_mean, out, s);
     if (r < 0) return cuda_fail("stats launch", cudaGetLastError());

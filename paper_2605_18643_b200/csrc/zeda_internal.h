@@ -96,8 +96,13 @@ namespace zeda {
 
 // ---- launchers (each returns the number of kernels it enqueued, or <0 on a launch error) ----
 int init_route_kernels(const zeda_moe *h);
-int launch_router_logits(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, cudaStream_t s);
-int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, const RouteOut &out, cudaStream_t s);
+// With n_parts == nullptr the logits are complete.  Otherwise the router may cut the reduction axis
+// into *n_parts slices (mid-sized batches on the tensor-core path): slice p then lies at
+// logits + p * T * n_cand, and launch_route_from_logits adds the slices in order.
+int launch_router_logits(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, cudaStream_t s,
+                         int *n_parts = nullptr);
+int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, const RouteOut &out, cudaStream_t s,
+                             int n_parts = 1);
 int launch_stats(const zeda_moe *h, const float *logits, const int32_t *topk_idx, int T, float *f,
                  float *p_mean, float *out, cudaStream_t s);
 int launch_experts_gemm1(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
@@ -105,7 +110,15 @@ int launch_experts_gemm2(const zeda_moe *h, int T, cudaStream_t s);
 int init_tile_kernels(zeda_moe *h);
 int router_split_pad(int n_cand);
 int init_router_tile(zeda_moe *h);
-int launch_router_logits_tile(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, cudaStream_t s);
+constexpr int kRouterMaxSplit = 4;
+// rows of n_cand floats that the workspace holds for router output (complete logits or their slices)
+inline long long router_part_rows(long long max_tokens) {
+    const long long cap = 9600;  // past this many tokens the unsplit grid covers the SMs already
+    const long long want = kRouterMaxSplit * max_tokens < cap ? kRouterMaxSplit * max_tokens : cap;
+    return max_tokens > want ? max_tokens : want;
+}
+int router_split_factor(const zeda_moe *h, int T);
+int launch_router_logits_tile(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, int split, cudaStream_t s);
 int launch_gather_rows(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
 int launch_experts_gemm1_tile(const zeda_moe *h, int T, cudaStream_t s);
 int launch_experts_gemm2_tile(const zeda_moe *h, int T, cudaStream_t s);

@@ -231,6 +231,28 @@ def test_tensor_core_router_path(zeda):
         run_layer(zeda, wl, token_ids=sample_tokens(T, 48, 1))
 
 
+@pytest.mark.parametrize("T,max_tokens", [(300, 300), (2500, 2500), (2500, 9000), (5000, 5000), (300, 20000)])
+def test_router_with_sliced_reduction_axis(zeda, T, max_tokens):
+    # mid-sized batches cut the router's reduction axis into 2 or 4 slices (as many as keep the grid
+    # within the SMs and the slices within the workspace); the top-K kernel adds them.  Routing from
+    # x must equal both the oracle's and the routing from the complete logits.
+    wl = inputs.tiny(seed=12, T=T, d=512, E=96, Z=40, K=4)
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev, max_tokens=max_tokens)
+    x = wl.x.to(dev)
+    l, idx, w, counts, offsets, perm, P = oracle_route(wl)
+    a = m.route(x)
+    check_route(a, idx, w, counts, offsets, perm, P)
+    b = m.route_from_logits(m.router_logits(x))
+    assert torch.equal(a["topk_idx"], b["topk_idx"]) and torch.equal(a["perm"], b["perm"])
+    # the statistics read complete logits, whichever way the routing before them got its own
+    f, p, _ = m.stats(x)
+    s = oracle.stats(l, idx, wl.E, wl.Z, alpha=1.0, group_w=1.0)
+    assert np.allclose(f.cpu().numpy(), s["f"], rtol=1e-5, atol=1e-7)
+    assert np.allclose(p.cpu().numpy(), s["P"], rtol=1e-4, atol=1e-7)
+    m.close()
+
+
 def test_streaming_expert_kernels(zeda):
     # the weight-streaming expert kernels (register MMAs) stay selectable by flag
     run_layer(zeda, inputs.tiny(seed=3), flags=1)
