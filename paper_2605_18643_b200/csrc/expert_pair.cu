@@ -22,9 +22,12 @@
 // Warp 2 (GEMM1): gather relay.  Warp 3 (GEMM2): TMA producer of the Hmid rows.  Warps 4-7:
 // epilogue.  Warps 8-11 (GEMM1): x-row gather.  Full barriers live in the leader CTA and count the
 // TMA bytes (and gather relays) of both CTAs; stage-empty and accumulator-full barriers are
-// signalled in both CTAs by multicast commits.  Every mbarrier wait is bounded; on expiry the CTA
-// records an error word, skips the rest of its work, and leaves through the common exit (cluster
-// barrier, TMEM free).
+// signalled in both CTAs by multicast commits.  The issuing warps (TMA producers, MMA issue, relay)
+// run their loops with all 32 lanes converged: every lane waits on the barrier, one elected lane
+// issues.  A loop confined to a single lane of a diverged warp costs about twice the cycles per
+// k-step, and that lane's instruction stream is what bounds a narrow tile.  Every mbarrier wait is
+// bounded; on expiry the CTA records an error word, skips the rest of its work, and leaves through
+// the common exit (cluster barrier, TMEM free).
 #include "tc_common.cuh"
 
 namespace zeda {
@@ -138,7 +141,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (weights)
-        if (lane == 0) {
+        {
             uint32_t it_count = 0;
             bool ok = true;
             Item nxt = {0, 0, 0, 0};  // the next item's description is fetched while this one is processed
@@ -150,25 +153,29 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 const uint32_t bytes = 2u * (uint32_t)(kATileBytes + (MODE == 2 ? half * kRowBytes : 0));
                 for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
                     const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
-                    if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag));
+                    if (!ok) break;
                     const uint32_t full = full0 + 8 * s;
                     const uint32_t sa = ring + s * kStageBytes;
-                    if (leader) mbar_expect_tx(bar_full + 8 * s, bytes);  // the TMA bytes of both CTAs
-                    if (MODE == 1)  // one box: 64 gate rows of block (2 mb + rank), then the 64 up rows of the same block
-                        tma_load_5d_pair(sa, &map_a, ks * kBlockK, 0, 0, 2 * it.mb + (int)rank, it.e, full);
-                    else
-                        tma_load_3d_pair(sa, &map_a, ks * kBlockK, 256 * it.mb + 128 * (int)rank, it.e, full);
+                    if (elect_one()) {
+                        if (leader) mbar_expect_tx(bar_full + 8 * s, bytes);  // the TMA bytes of both CTAs
+                        if (MODE == 1)  // one box: 64 gate rows of block (2 mb + rank), then the 64 up rows of the same block
+                            tma_load_5d_pair(sa, &map_a, ks * kBlockK, 0, 0, 2 * it.mb + (int)rank, it.e, full);
+                        else
+                            tma_load_3d_pair(sa, &map_a, ks * kBlockK, 256 * it.mb + 128 * (int)rank, it.e, full);
+                    }
+                    __syncwarp();
                 }
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 if (!*abort_flag) atomicExch(&meta[kMetaError], 11);
                 s_abort = 1;
             }
         }
     } else if (MODE == 2 && warp == 3) {
         // ------------------------------------------------------------------ TMA producer of the Hmid rows (GEMM2)
-        // A second issuing thread: one thread cannot issue the loads of both operands fast enough.
-        if (lane == 0) {
+        // A second issuing warp: one cannot issue the loads of both operands fast enough.
+        {
             uint32_t it_count = 0;
             bool ok = true;
             Item nxt = {0, 0, 0, 0};  // the next item's description is fetched while this one is processed
@@ -180,28 +187,32 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 const int brow0 = (int)rank * half;  // first tile column / pair row this CTA loads
                 for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
                     const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
-                    if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag));
+                    if (!ok) break;
                     const uint32_t full = full0 + 8 * s;
                     const uint32_t sb = ring + s * kStageBytes + kATileBytes;
-                    int b = 0;
+                    if (elect_one()) {
+                        int b = 0;
 #pragma unroll
-                    for (int lvl = 0; lvl < 4; ++lvl) {
-                        const int rows = 128 >> lvl;
-                        if (rows <= HALF_MAX && half - b >= rows) {
-                            tma_load_2d_pair(sb + b * kRowBytes, &maps_b.m[lvl], ks * kBlockK, it.pos0 + brow0 + b, full);
-                            b += rows;
+                        for (int lvl = 0; lvl < 4; ++lvl) {
+                            const int rows = 128 >> lvl;
+                            if (rows <= HALF_MAX && half - b >= rows) {
+                                tma_load_2d_pair(sb + b * kRowBytes, &maps_b.m[lvl], ks * kBlockK, it.pos0 + brow0 + b, full);
+                                b += rows;
+                            }
                         }
                     }
+                    __syncwarp();
                 }
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 if (!*abort_flag) atomicExch(&meta[kMetaError], 16);
                 s_abort = 1;
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA)
-        if (leader && lane == 0) {
+        if (leader) {
             uint32_t tile_count = 0;
             uint32_t s = 0, ph = 0;  // ring stage of the next k-step and the parity of its use
             // descriptors of stage 0; stage s is (s * kStageBytes) >> 4 further in the address field
@@ -215,24 +226,30 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 const int n_cols = ((it.n + 31) >> 5) << 5;
                 const uint32_t idesc = instr_desc_pair(n_cols);
                 const uint32_t buf = tile_count & 1u, tph = (tile_count >> 1) & 1u;
-                if (!mbar_wait(bar_tempty + 8 * buf, tph ^ 1u, abort_flag)) { ok = false; break; }
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * buf, tph ^ 1u, abort_flag));
+                if (!ok) break;
                 tc_fence_after();
                 const uint32_t d = tmem_base + buf * kAccCols;
                 for (int ks = 0; ks < k_steps; ++ks) {
-                    if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph, abort_flag));
+                    if (!ok) break;
                     tc_fence_after();
                     const uint64_t a = a0 + (uint64_t)(s * (kStageBytes >> 4));
                     const uint64_t b = b0 + (uint64_t)(s * (kStageBytes >> 4));
+                    if (elect_one()) {  // always the same lane: a commit covers the MMAs of the thread that issues it
 #pragma unroll
-                    for (int k = 0; k < kBlockK / 16; ++k)  // +32 bytes per 16-element k slice inside the swizzle row
-                        umma_bf16_pair(d, a + 2 * k, b + 2 * k, idesc, (ks | k) ? 1u : 0u);
-                    umma_commit_pair(bar_empty + 8 * s);  // the stage is free in both CTAs once these MMAs have read it
+                        for (int k = 0; k < kBlockK / 16; ++k)  // +32 bytes per 16-element k slice inside the swizzle row
+                            umma_bf16_pair(d, a + 2 * k, b + 2 * k, idesc, (ks | k) ? 1u : 0u);
+                        umma_commit_pair(bar_empty + 8 * s);  // the stage is free in both CTAs once these MMAs have read it
+                    }
+                    __syncwarp();
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit_pair(bar_tfull + 8 * buf);    // accumulators complete in both CTAs
+                if (elect_one()) umma_commit_pair(bar_tfull + 8 * buf);    // accumulators complete in both CTAs
+                __syncwarp();
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 if (!*abort_flag) atomicExch(&meta[kMetaError], 12);
                 s_abort = 1;
             }
@@ -241,17 +258,19 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         // ------------------------------------------------------------------ gather relay (GEMM1)
         // cp.async can only signal an mbarrier of its own CTA: this thread forwards "this CTA's
         // gathered rows of stage s have landed" to the leader's full barrier.
-        if (lane == 0) {
+        {
             uint32_t it_count = 0;
             bool ok = true;
             for (long long item = first; item < n_items && ok; item += stride) {
                 for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
                     const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
-                    if (!mbar_wait(bar_gfull + 8 * s, ph, abort_flag)) { ok = false; break; }
-                    mbar_arrive_cluster(full0 + 8 * s);
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_gfull + 8 * s, ph, abort_flag));
+                    if (!ok) break;
+                    if (elect_one()) mbar_arrive_cluster(full0 + 8 * s);
+                    __syncwarp();
                 }
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 if (!*abort_flag) atomicExch(&meta[kMetaError], 15);
                 s_abort = 1;
             }

@@ -36,6 +36,13 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
+// True in exactly one lane of a converged warp (the same lane on every call with a full warp).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+
 // Bounded wait: false if the limit passed or another role already gave up.  The common case (the
 // phase completes within a few thousand polls) reads no timer at all; after that the SM's own
 // cycle counter bounds the wait.
