@@ -203,6 +203,25 @@ slot_hist_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real,
 // ---------------------------------------------------------------------------------------------
 constexpr int kScanSlabInts = 8192;  // 32 KB of CTA histograms per slab of the expert scan
 
+// Copies n ints from global to shared memory with sixteen loads in flight per thread: a plain
+// load-store loop issues its loads one L2 round trip after another (the store waits for the load).
+__device__ __forceinline__ void stage_ints(int32_t *__restrict__ dst, const int32_t *__restrict__ src, int n) {
+    constexpr int kInFlight = 16;
+    for (int i0 = threadIdx.x; i0 < n; i0 += kInFlight * blockDim.x) {
+        int32_t v[kInFlight];
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            const int i = i0 + u * blockDim.x;
+            v[u] = i < n ? __ldg(src + i) : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) {
+            const int i = i0 + u * blockDim.x;
+            if (i < n) dst[i] = v[u];
+        }
+    }
+}
+
 struct ScanShared {
     int32_t cnt[kMaxCand];
     int32_t off[kMaxCand + 1];
@@ -216,7 +235,8 @@ struct ScanShared {
 __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, int total_slots,
                                                    int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
                                                    int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
-                                                   const WorkLists &wl, bool write_global = true) {
+                                                   const WorkLists &wl, bool write_global = true,
+                                                   int list_part = 0, int list_parts = 1) {
     if (threadIdx.x < 32) {
         // warp 0 scans the three per-expert sequences in steps of 32 with shuffle prefix sums
         int base_off = 0, base_chunk = 0, base_tile = 0, base_ptile = 0, active = 0, max_rows = 0;
@@ -269,16 +289,20 @@ __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, i
         }
     }
     __syncthreads();
-    if (!write_global) return;  // (uniform over the CTA)
-    for (int e = threadIdx.x; e < n_real; e += blockDim.x) {
-        if (counts) counts[e] = sh.cnt[e];
-        offsets[e] = sh.off[e];
+    if (write_global) {  // (uniform over the CTA)
+        for (int e = threadIdx.x; e < n_real; e += blockDim.x) {
+            if (counts) counts[e] = sh.cnt[e];
+            offsets[e] = sh.off[e];
+        }
+        if (threadIdx.x == 0) offsets[n_real] = sh.off[n_real];
     }
-    if (threadIdx.x == 0) offsets[n_real] = sh.off[n_real];
+    // Work lists: every CTA that runs this scan holds the same prefix sums, so the CTAs share the
+    // filling (part list_part of list_parts); a CTA outside that sharing passes list_parts = 0.
+    if (list_parts <= 0) return;
     // work lists: entry i belongs to the expert whose first-entry index is the last one <= i
     auto fill = [&](const int32_t *first, int rows, int32_t *list_expert, int32_t *list_row0) {
         const int total = first[n_real];
-        for (int i = threadIdx.x; i < total; i += blockDim.x) {
+        for (int i = list_part * blockDim.x + threadIdx.x; i < total; i += list_parts * blockDim.x) {
             int lo = 0, hi = n_real;  // invariant: first[lo] <= i < first[hi]
             while (hi - lo > 1) {
                 const int mid = (lo + hi) >> 1;
@@ -463,8 +487,9 @@ slot_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real
 // ---------------------------------------------------------------------------------------------
 // Counting sort, passes 2 + 3 in one launch (used while the CTA histograms are few): every CTA
 // sums the histogram columns itself (pairs of each expert in earlier CTAs, and in all CTAs), scans
-// the expert totals, and places its slots as above.  CTA 0 also publishes counts, offsets, the
-// counters and the work lists.  Saves a launch and the single-CTA scan between two short kernels.
+// the expert totals, and places its slots as above.  CTA 0 also publishes counts, offsets and the
+// counters; the work lists are filled by all CTAs, a share each.  Saves a launch and the single-CTA
+// scan between two short kernels.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kPlaceWarps * 32)
 slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real, int nblk,
@@ -488,7 +513,7 @@ slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n
         const int nb = min(slab_blocks, nblk - b0);
         const int32_t *g = block_hist + (size_t)b0 * n_real;
         __syncthreads();
-        for (int i = threadIdx.x; i < nb * n_real; i += blockDim.x) slab[i] = __ldg(g + i);
+        stage_ints(slab, g, nb * n_real);
         __syncthreads();
         for (int e = threadIdx.x; e < n_real; e += blockDim.x) {
             int before = 0, total = 0;
@@ -502,7 +527,7 @@ slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n
         }
     }
     __syncthreads();
-    finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, wl, blockIdx.x == 0);
+    finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, wl, blockIdx.x == 0, blockIdx.x, gridDim.x);
     __syncthreads();
     const int s0 = blockIdx.x * kSortTokens * K;
     const int s1 = min(T * K, s0 + kSortTokens * K);
@@ -666,6 +691,7 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
     do {                                               \
         if (n_cand <= 64) { CALL(2); }                 \
         else if (n_cand <= 128) { CALL(4); }           \
+        else if (n_cand <= 192) { CALL(6); }           \
         else if (n_cand <= 256) { CALL(8); }           \
         else { CALL(16); }                             \
     } while (0)
