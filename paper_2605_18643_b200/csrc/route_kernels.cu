@@ -655,6 +655,11 @@ int init_route_kernels(const zeda_moe *h) {
     if (smem > 48 * 1024 &&
         cudaFuncSetAttribute(router_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return -1;
+    // placement CTAs: static scan state plus (per-warp positions, bases, a histogram slab) pass 48 KB
+    // together when there are many experts
+    const int place_smem = (int)sizeof(int32_t) * ((kPlaceWarps + 1) * kMaxCand + kScanSlabInts);
+    if (cudaFuncSetAttribute(slot_scan_place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, place_smem) != cudaSuccess)
+        return -1;
     return 0;
 }
 

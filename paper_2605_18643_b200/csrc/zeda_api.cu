@@ -88,7 +88,11 @@ size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+thread_local cudaError_t t_launch_error = cudaSuccess;
+
 zeda_status_t cuda_fail(const char *what, cudaError_t e) {
+    if (e == cudaSuccess) e = t_launch_error;  // a launch that failed earlier in this call
+    t_launch_error = cudaSuccess;
     set_error("%s: %s", what, cudaGetErrorString(e));
     return ZEDA_ERR_CUDA;
 }
@@ -157,6 +161,11 @@ zeda_status_t forward_device(zeda_moe_t *h, const __nv_bfloat16 *x, int T, __nv_
 }
 
 }  // namespace
+
+void note_launch_error(cudaError_t e) {
+    if (t_launch_error == cudaSuccess) t_launch_error = e;
+}
+
 }  // namespace zeda
 
 using namespace zeda;

@@ -129,6 +129,9 @@ int launch_wait_selftest(const zeda_moe *h, long long limit_cycles, cudaStream_t
 int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s);
 
 void set_error(const char *fmt, ...);
+// remembers the error of a failed kernel launch for the status message of the API call (the runtime's
+// own "last error" may have been read and cleared by a later launch check)
+void note_launch_error(cudaError_t e);
 
 // ---- programmatic dependent launch ------------------------------------------------------------
 // The kernels of one forward pass are launched back to back on one stream.  Launched with the
@@ -154,7 +157,9 @@ inline cudaError_t launch_kernel(bool pdl, void (*kernel)(KArgs...), dim3 grid, 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+    if (e != cudaSuccess) note_launch_error(e);
+    return e;
 }
 #endif
 

@@ -347,6 +347,15 @@ def test_routing_with_many_sort_blocks(zeda):
     m.close()
 
 
+@pytest.mark.parametrize("T", [40, 600])
+def test_maximum_candidates_and_top_k(zeda, T):
+    # the limits of the interface: N + N_Z = 512 candidates (16 logits per lane in the top-K warp,
+    # four candidate tiles in the tensor-core router) and K = 16 slots per token
+    wl = inputs.tiny(seed=13, T=T, d=256, He=128, E=384, Z=128, K=16)
+    err, (P, U, zs) = run_layer(zeda, wl, token_ids=sample_tokens(T, 24, 6))
+    assert P + zs == T * 16 and zs > 0 and U > 100
+
+
 # ---------------------------------------------------------------------------------- second model shape
 
 def test_glm_shaped_layer_and_net_point(zeda):
