@@ -3,6 +3,8 @@
 Bars: routing indices, per-expert counts, offsets, permutation and P bit-exact; routing weights
 within fp32 rounding (rel 1e-5); layer output rel-L2 <= 1e-2 and max-abs <= 5e-2 * RMS(y).
 """
+import copy
+
 import numpy as np
 import pytest
 import torch
@@ -77,7 +79,8 @@ def run_layer(zeda, wl, token_ids=None, gate_mode=0, expert_kind=0, flags=0, che
     if check_routing:
         l, idx, w, counts, offsets, perm, P = oracle_route(wl, gate_mode)
         gl = m.router_logits(x).cpu().numpy()
-        assert np.max(np.abs(gl.astype(np.float64) - l.astype(np.float64))) < 2e-5
+        # fp32 accumulation over d products: the bar grows with d beyond the spec width
+        assert np.max(np.abs(gl.astype(np.float64) - l.astype(np.float64))) < 2e-5 * max(1.0, wl.d / 2048)
         check_route(m.route(x), idx, w, counts, offsets, perm, P)
     y = m.forward(x)
     torch.cuda.synchronize()
@@ -343,7 +346,13 @@ def test_routing_with_many_sort_blocks(zeda):
     dev = torch.device("cuda:0")
     m = zeda.from_workload(wl, dev)
     l, idx, w, counts, offsets, perm, P = oracle_route(wl)
-    check_route(m.route(wl.x.to(dev)), idx, w, counts, offsets, perm, P)
+    x = wl.x.to(dev)
+    check_route(m.route(x), idx, w, counts, offsets, perm, P)
+    ids = sample_tokens(wl.T, 48, 9)
+    y = m.forward(x)
+    torch.cuda.synchronize()
+    y_ref, _, _ = oracle_forward(wl, ids)
+    check_y(y[torch.as_tensor(ids, device=dev, dtype=torch.long)], y_ref)
     m.close()
 
 
@@ -354,6 +363,42 @@ def test_maximum_candidates_and_top_k(zeda, T):
     wl = inputs.tiny(seed=13, T=T, d=256, He=128, E=384, Z=128, K=16)
     err, (P, U, zs) = run_layer(zeda, wl, token_ids=sample_tokens(T, 24, 6))
     assert P + zs == T * 16 and zs > 0 and U > 100
+
+
+def test_one_handle_many_batch_sizes(zeda):
+    # one handle (workspace sized for the largest batch) serves calls of very different sizes in a
+    # row: nothing of an earlier call (work lists, counters, histograms) may leak into the next
+    base = inputs.tiny(seed=14, T=900)
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(base, dev, max_tokens=900)
+    for T in (900, 5, 300, 64, 1, 257, 900):
+        wl = copy.copy(base)                      # the same layer on the first T tokens
+        wl.x, wl.T = base.x[:T].contiguous(), T
+        x = wl.x.to(dev)
+        l, idx, w, counts, offsets, perm, P = oracle_route(wl)
+        check_route(m.route(x), idx, w, counts, offsets, perm, P)
+        y = m.forward(x)
+        torch.cuda.synchronize()
+        ids = sample_tokens(T, min(T, 32), T)
+        y_ref, _, _ = oracle_forward(wl, ids)
+        check_y(y[torch.as_tensor(ids, device=dev, dtype=torch.long)], y_ref)
+    m.close()
+
+
+@pytest.mark.parametrize("E,Z,K", [(1, 1, 2), (1, 0, 1), (8, 4, 1), (2, 30, 8)])
+def test_degenerate_expert_sets(zeda, E, Z, K):
+    # one normal expert; no zero expert at all with K = 1; a single slot per token; far more zero
+    # experts than normal ones
+    for T in (33, 300):
+        wl = inputs.tiny(seed=15, T=T, E=E, Z=Z, K=K, zero_fraction=None)
+        run_layer(zeda, wl, token_ids=sample_tokens(T, 24, 7))
+
+
+def test_wide_model_and_expert_dimensions(zeda):
+    # many k-steps per work item in both GEMMs (d = 4096: 64 k-steps in GEMM1; H_e = 2048: 32 in
+    # GEMM2) and many weight-row blocks
+    wl = inputs.tiny(seed=16, T=320, d=4096, He=2048, E=4, Z=2, K=2)
+    run_layer(zeda, wl, token_ids=sample_tokens(320, 16, 8))
 
 
 # ---------------------------------------------------------------------------------- second model shape
