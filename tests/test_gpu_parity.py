@@ -113,6 +113,13 @@ def test_tiny_gate_modes_and_copy_experts(zeda, gate_mode, expert_kind):
     run_layer(zeda, inputs.tiny(seed=1), gate_mode=gate_mode, expert_kind=expert_kind)
 
 
+@pytest.mark.parametrize("gate_mode,expert_kind", [(1, 0), (2, 0), (0, 1), (2, 1)])
+def test_gate_modes_and_copy_experts_on_the_large_batch_kernels(zeda, gate_mode, expert_kind):
+    # T > 128: separate top-K kernel, tensor-core router, multi-CTA counting sort
+    wl = inputs.tiny(seed=3, T=300)
+    run_layer(zeda, wl, token_ids=sample_tokens(300, 40, 2), gate_mode=gate_mode, expert_kind=expert_kind)
+
+
 def test_tiny_static_layer_z0(zeda):
     wl = inputs.tiny(seed=2, Z=0, zero_fraction=None)
     err, (P, U, zs) = run_layer(zeda, wl)
