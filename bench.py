@@ -32,7 +32,7 @@ METRIC = "MoE-layer tokens/s"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (expert GEMM1),
 # from the ncu captures summarised under profiles/ (same workloads, same kernel build)
-NCU_TRAFFIC_BYTES = {"prefill": 621.3e6, "decode": 742.4e6}
+NCU_TRAFFIC_BYTES = {"prefill": 624.8e6, "decode": 740.9e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
