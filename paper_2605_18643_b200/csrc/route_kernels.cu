@@ -36,11 +36,21 @@ router_logits_kernel(const __nv_bfloat16 *__restrict__ x, const float *__restric
     const int t0 = blockIdx.x * kTok;
     const int nt = min(kTok, T - t0);
     const int vec_per_row = d / 8;
-    for (int i = threadIdx.x; i < kTok * vec_per_row; i += blockDim.x) {
-        const int r = i / vec_per_row, c = i % vec_per_row;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (r < nt) v = __ldg(reinterpret_cast<const uint4 *>(x + (size_t)(t0 + r) * d) + c);
-        reinterpret_cast<uint4 *>(xs + (size_t)r * d)[c] = v;
+    // eight 16-byte loads in flight per thread (a plain load-store loop waits for each load in turn)
+    for (int i0 = threadIdx.x; i0 < kTok * vec_per_row; i0 += 8 * blockDim.x) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + u * blockDim.x;
+            const int r = i / vec_per_row, c = i % vec_per_row;
+            v[u] = make_uint4(0, 0, 0, 0);
+            if (i < kTok * vec_per_row && r < nt) v[u] = __ldg(reinterpret_cast<const uint4 *>(x + (size_t)(t0 + r) * d) + c);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + u * blockDim.x;
+            if (i < kTok * vec_per_row) reinterpret_cast<uint4 *>(xs + (size_t)(i / vec_per_row) * d)[i % vec_per_row] = v[u];
+        }
     }
     __syncthreads();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
