@@ -514,6 +514,21 @@ slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n
     int32_t *base = pos + kPlaceWarps * n_real;
     int32_t *slab = base + n_real;         // [kScanSlabInts]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // this warp's slots, fetched now (their latency passes under the histogram sums below): slot
+    // w0 + 32 u + lane in e_reg[u], -1 for zero-expert slots and beyond the end
+    constexpr int kSlotRegs = kSortTokens * kMaxTopK / kPlaceWarps / 32;
+    const int s0 = blockIdx.x * kSortTokens * K;
+    const int s1 = min(T * K, s0 + kSortTokens * K);
+    const int per_warp = ((kSortTokens * K + kPlaceWarps - 1) / kPlaceWarps + 31) / 32 * 32;
+    const int w0 = s0 + warp * per_warp;
+    const int w1 = min(s1, w0 + per_warp);
+    int e_reg[kSlotRegs];
+#pragma unroll
+    for (int u = 0; u < kSlotRegs; ++u) {
+        const int s = w0 + 32 * u + lane;
+        int e = (32 * u < per_warp && s < w1) ? __ldg(topk_idx + s) : -1;
+        e_reg[u] = e >= n_real ? -1 : e;
+    }
     for (int i = threadIdx.x; i < kPlaceWarps * n_real; i += blockDim.x) pos[i] = 0;
     for (int e = threadIdx.x; e < n_real; e += blockDim.x) { base[e] = 0; sh.cnt[e] = 0; }
     // column sums of the CTA histograms: staged slab by slab with independent coalesced loads (a
@@ -539,16 +554,12 @@ slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n
     __syncthreads();
     finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, wl, blockIdx.x == 0, blockIdx.x, gridDim.x);
     __syncthreads();
-    const int s0 = blockIdx.x * kSortTokens * K;
-    const int s1 = min(T * K, s0 + kSortTokens * K);
-    const int per_warp = ((kSortTokens * K + kPlaceWarps - 1) / kPlaceWarps + 31) / 32 * 32;
-    const int w0 = s0 + warp * per_warp;
-    const int w1 = min(s1, w0 + per_warp);
     int32_t *mine = pos + warp * n_real;
     const unsigned lt = (1u << lane) - 1u;
-    for (int s = w0 + lane; s - lane < w1; s += 32) {
-        int e = (s < w1) ? topk_idx[s] : -1;
-        if (e >= n_real) e = -1;
+#pragma unroll
+    for (int u = 0; u < kSlotRegs; ++u) {
+        if (w0 + 32 * u >= w1 || 32 * u >= per_warp) break;  // (uniform over the warp)
+        const int e = e_reg[u];
         const unsigned grp = __match_any_sync(kFull, e);
         if (e >= 0 && (grp & lt) == 0) mine[e] += __popc(grp);
         __syncwarp();
@@ -563,10 +574,12 @@ slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n
         }
     }
     __syncthreads();
-    for (int s = w0 + lane; s - lane < w1; s += 32) {
-        int e = (s < w1) ? topk_idx[s] : -1;
+#pragma unroll
+    for (int u = 0; u < kSlotRegs; ++u) {
+        if (w0 + 32 * u >= w1 || 32 * u >= per_warp) break;  // (uniform over the warp)
+        const int s = w0 + 32 * u + lane;
+        const int e = e_reg[u];
         const bool in_range = s < w1;
-        if (e >= n_real) e = -1;
         const unsigned grp = __match_any_sync(kFull, e);
         int p = -1;
         if (e >= 0) p = mine[e] + __popc(grp & lt);
