@@ -123,7 +123,10 @@ zeda_status_t zeda_route_from_logits(zeda_moe_t *h, const float *logits, int32_t
                                      int32_t *expert_offsets, int32_t *perm, int32_t *n_pairs,
                                      void *stream);
 
-/* Test entry: the fp32 router logits x * router_w^T + bias, dev [T, N+N_Z]. */
+/* Test entry: the fp32 router logits x * router_w^T + bias, dev [T, N+N_Z].  zeda_route and
+ * zeda_moe_forward compute the same sums, for mid-sized batches (256 <= T, up to a few thousand
+ * tokens) in two or four slices of the reduction axis that are added afterwards: their logits can
+ * differ from these in the last bits (fp32 addition order), never in the exact products. */
 zeda_status_t zeda_router_logits(zeda_moe_t *h, const void *x, int32_t T, float *logits, void *stream);
 
 /* Layer forward, Eq. 1 (Eq. 7 / Appendix B through the configured modes).
