@@ -2,10 +2,12 @@
 """Benchmark of the zero-expert MoE layer forward (one step = one zeda_moe_forward call over one
 batch of synthetic tokens: router, top-K, compaction, grouped SwiGLU experts, combine).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload decode|prefill|sweep25|...]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload prefill|decode|net|glm|sweep25|stack|...]
     python bench.py --impl reference ...      # the CPU oracle, timed on the host cores
 
-Prints ONE JSON line.  With N > 1 (launched by torch.distributed.run) every rank is a data-parallel
+Prints ONE JSON line.  The default workload is the prefill batch (T = 8192) of the Qwen3-30B-A3B-shaped
+layer; its line also carries, as nested objects, the decode batch (T = 64) on the same layer, the
+static top-K layer (Z = 0) and the NET layer (Z = 0, K/2) run through the same kernels.  With N > 1 (launched by torch.distributed.run) every rank is a data-parallel
 replica of the layer with its own token batch; there is no collective on the data path.
 """
 from __future__ import annotations
@@ -30,10 +32,11 @@ from paper_2605_18643_b200 import flops, inputs
 
 METRIC = "MoE-layer tokens/s"
 UNIT = "tokens/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (expert GEMM1),
-# from the ncu captures summarised under profiles/ (same workloads, same kernel build)
-NCU_TRAFFIC_BYTES = {"prefill": 624.8e6, "decode": 740.9e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+L2_NOTE = "256 MiB written, then 256 MiB read, between timed steps (outside the event pairs)"
+# sources of the dominant kernel (expert GEMM1 + SwiGLU): the ncu traffic figures are only valid for
+# the build they were captured on
+GEMM_SOURCES = ("expert_pair.cu", "tc_common.cuh")
 
 
 def load_peaks():
@@ -45,6 +48,35 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
+def kernel_source_id():
+    """Short hash of the expert kernels' sources: ties an ncu traffic figure to the build it was taken on."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in GEMM_SOURCES:
+        with open(os.path.join(ROOT, "paper_2605_18643_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:12]
+
+
+def ncu_traffic_bytes(workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the
+    line `<workload> <bytes> <source id>` of profiles/gemm1_dram_traffic.txt (written beside the
+    ncu summary it comes from).  None when there is no line for this workload or the kernel's
+    sources have changed since the capture."""
+    p = os.path.join(ROOT, "profiles", "gemm1_dram_traffic.txt")
+    if not os.path.exists(p):
+        return None
+    sid = kernel_source_id()
+    for line in open(p):
+        f = line.split()
+        if len(f) >= 3 and not line.startswith("#") and f[0] == workload and f[2] == sid:
+            return float(f[1])
+    return None
+
+
+GLM_SHAPE = dict(d=2048, He=1536, E=64, Z=32, K=4)   # N, K, N_Z from the paper's table of adapted models; d, H_e free
+
+
 def make_workload(name: str):
     if name == "decode":
         return inputs.decode()
@@ -52,6 +84,10 @@ def make_workload(name: str):
         return inputs.prefill()
     if name == "tiny":
         return inputs.tiny()
+    if name == "net":      # the paper's iso-FLOP static baseline: no zero experts, K/2 slots
+        return net_reference(inputs.prefill())
+    if name == "glm":      # second adapted model's expert counts at the prefill size
+        return inputs.make_layer("glm", T=8192, zero_fraction=0.5, zipf_s=1.1, **GLM_SHAPE)
     if name.startswith("sweep"):
         return inputs.sweep_point(int(name[5:]) / 100.0)
     if name.startswith("prefill_f"):   # zero-fraction sweep at the prefill size
@@ -60,12 +96,19 @@ def make_workload(name: str):
     raise SystemExit("unknown workload " + name)
 
 
-def workload_config(wl, name, extra=None):
-    c = {"workload": name, "T": wl.T, "d": wl.d, "d_expert": wl.He, "n_real": wl.E, "n_zero": wl.Z,
-         "top_k": wl.K, "zero_slot_fraction": round(wl.zero_fraction, 4), "seed": 0}
-    if extra:
-        c.update(extra)
-    return c
+def net_reference(wl):
+    """NET (Section 3.1): the static layer with half the slots, K/2, and no zero experts, on the same
+    x, expert weights, normal router rows and normal-expert bias."""
+    import dataclasses
+    st = inputs.static_reference(wl)
+    return dataclasses.replace(st, name=wl.name + "_net", K=max(1, wl.K // 2))
+
+
+def workload_config(wl, name, P, U, world):
+    """The `config` object of the JSON line; identical for both arms (P and U follow from the routing)."""
+    return {"workload": name, "T": wl.T, "d": wl.d, "d_expert": wl.He, "n_real": wl.E, "n_zero": wl.Z,
+            "top_k": wl.K, "zero_slot_fraction": round(wl.zero_fraction, 4), "seed": 0, "P": int(P), "U": int(U),
+            "l2": L2_NOTE, "parallelism": "dp%d replicas, no collective" % world}
 
 
 class ClockSampler:
@@ -141,31 +184,41 @@ def oracle_tokens_per_s(wl, sample_tokens: int, seed: int = 0, min_seconds: floa
     return n * passes / dt, dt, oracle.num_threads(), "%s, %d passes" % (what, passes)
 
 
+def oracle_pairs(wl):
+    """P and U of the workload from the oracle's routing of every token (no expert math)."""
+    import oracle
+    bias = None if wl.router_bias is None else wl.router_bias.numpy()
+    _, idx, _ = oracle.forward(inputs.bits(wl.x), wl.router_w.numpy(), bias, inputs.bits(wl.w_gate_up),
+                               inputs.bits(wl.w_down), wl.E, wl.Z, wl.K, want_y=False)
+    counts, _, _, P = oracle.compact(idx, wl.E)
+    return P, int((counts > 0).sum())
+
+
 def run_reference(args):
-    """--impl reference: the CPU oracle on the host cores, same metric and workload."""
+    """--impl reference: the CPU oracle on the host cores, same metric, workload and config.  Each
+    step is the oracle, as it stands, on a bounded seeded sample of the workload's tokens."""
     rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
     if rank != 0:
         return
     wl = make_workload(args.workload)
+    P, U = oracle_pairs(wl)
     sample = 64 if wl.T > 64 else wl.T
-    for _ in range(min(args.warmup, 1)):
+    for _ in range(args.warmup):
         oracle_tokens_per_s(wl, sample)
-    times, tps = [], []
-    steps = max(1, min(args.steps, 5))
-    info = None
-    for _ in range(steps):
+    total, info = 0.0, None
+    for _ in range(args.steps):
         v, dt, cores, desc = oracle_tokens_per_s(wl, sample)
-        times.append(dt)
-        tps.append(v)
+        total += dt
         info = (cores, desc)
-    total = sum(times)
-    value = sample * steps / total
+    value = sample * args.steps / total
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
-        "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * total / steps, "higher_is_better": True,
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(wl, args.workload, {"note": "each step = the oracle on a bounded token sample"}),
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": info[0], "kind": "oracle", "sample": info[1]},
+        "config": workload_config(wl, args.workload, P, U, world),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": info[0], "kind": "oracle",
+                         "sample": "each step = the oracle on %s" % info[1]},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -344,15 +397,141 @@ def run_stack(args, peaks, peaks_kind, dev, world, rank, barrier, dist):
         m.close()
 
 
+class DeviceWeights:
+    """Device copies of expert weights, shared between the handles of one run (the zero-expert layer,
+    its static reference, the decode batch on the same layer): 1.2 GB is copied once."""
+
+    def __init__(self, dev):
+        self.dev = dev
+        self.cache = {}
+
+    def handle(self, zeda, wl, max_tokens=None):
+        key = (wl.w_gate_up.data_ptr(), wl.w_down.data_ptr())
+        if key not in self.cache:
+            self.cache[key] = (wl.w_gate_up.to(self.dev).contiguous(), wl.w_down.to(self.dev).contiguous())
+        wgu, wd = self.cache[key]
+        bias = None if wl.router_bias is None else wl.router_bias.to(self.dev).contiguous()
+        return zeda.ZedaMoE(wl.router_w.to(self.dev).contiguous(), bias, wgu, wd, wl.E, wl.Z, wl.K, max_tokens or wl.T)
+
+
+def gemm1_roofline(wl, P, U, kernel_ms, peaks, peaks_kind, workload):
+    """Roofline object of the dominant kernel (expert GEMM1 + SwiGLU).  Algorithmic bytes: gate and up
+    weights of the U active experts + the x rows read + the intermediate written; algorithmic FLOPs:
+    4 d H_e per pair.  The kernel is timed by stage events inside the step, back to back with the other
+    kernels, so the tensor peak it is held against is the sustained one (burst beside it)."""
+    hbm = peaks["hbm_gbs"] * 1e9
+    burst = peaks["bf16_tflops"]
+    sustained = peaks.get("bf16_tflops_sustained", burst)
+    g1_bytes = U * 2 * wl.He * wl.d * 2 + wl.T * wl.d * 2 + P * wl.He * 2
+    g1_flops = 4 * P * wl.d * wl.He
+    g1_s = kernel_ms * 1e-3
+    if g1_bytes / hbm >= g1_flops / (sustained * 1e12):
+        roof = {"bound": "hbm", "achieved": g1_bytes / g1_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roof = {"bound": "tensor", "achieved": g1_flops / g1_s / 1e12, "peak": sustained, "unit": "TFLOP/s",
+                "peak_kind": "sustained (kernel timed inside the step)", "peak_burst": burst,
+                "frac_of_burst": g1_flops / g1_s / 1e12 / burst}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof.update(traffic=ncu_traffic_bytes(workload), kernel="expert GEMM1 + SwiGLU (expert_gemm_pair_kernel<1,..>)",
+                peak_source=peaks_kind, algorithmic_bytes=g1_bytes, algorithmic_flops=g1_flops, kernel_ms=kernel_ms)
+    return roof
+
+
+def layer_roofline(wl, P, U, ms_per_step, peaks, peaks_kind):
+    hbm = peaks["hbm_gbs"] * 1e9
+    burst = peaks["bf16_tflops"]
+    sustained = peaks.get("bf16_tflops_sustained", burst)
+    n_cand = wl.E + wl.Z
+    t_roof, t_flop, t_mem = flops.layer_roofline_seconds(wl.T, wl.d, wl.He, n_cand, P, U, burst * 1e12, hbm)
+    t_roof_s, t_flop_s, _ = flops.layer_roofline_seconds(wl.T, wl.d, wl.He, n_cand, P, U, sustained * 1e12, hbm)
+    return {"t_roof_us": t_roof * 1e6, "t_flop_us": t_flop * 1e6, "t_hbm_us": t_mem * 1e6,
+            "frac": t_roof / (ms_per_step * 1e-3), "peak_source": peaks_kind,
+            "t_flop_us_sustained": t_flop_s * 1e6, "t_roof_us_sustained": t_roof_s * 1e6,
+            "frac_sustained": t_roof_s / (ms_per_step * 1e-3)}
+
+
+def measure_layer(zeda, weights, wl, x_cpu, args, flush, barrier, dist, dev, e2e=True, static=True, net=False):
+    """Times one workload: the step itself, its stages, the host-buffer entry point, and the same
+    kernels on the static (Z = 0) and NET (Z = 0, K/2) reference layers.  Every rank runs this; the
+    timings returned are maxima over the ranks."""
+    m = weights.handle(zeda, wl)
+    x = x_cpu.to(dev)
+    y = torch.empty_like(x)
+    total_ms, _ = time_forward(m, x, y, args.steps, args.warmup, flush, barrier)
+    P, U, zero_slots, launches = m.last_counters()
+    # the same steps again with stage events on the stream: duration of every stage
+    m.set_profiling(True)
+    stage = np.zeros(5)
+    for i in range(args.steps):
+        flush.zero_()
+        m.forward(x, y)
+        stage += np.array(m.stage_ms())
+    stage /= args.steps
+    m.set_profiling(False)
+    e2e_s = 0.0
+    if e2e:
+        # end to end through the host-buffer entry point: H2D of x and D2H of y inside the timed region
+        x_pin = x_cpu.pin_memory()
+        y_pin = torch.empty_like(x_pin).pin_memory()
+        for _ in range(args.warmup):
+            flush.zero_()
+            m.forward_host(x_pin, y_pin)
+        barrier()
+        torch.cuda.synchronize()
+        for i in range(args.steps):
+            flush.zero_()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            m.forward_host(x_pin, y_pin)
+            e2e_s += time.perf_counter() - t0
+        barrier()
+    m.close()
+    refs = {}
+    if static and wl.Z > 0:
+        todo = [("static_reference", inputs.static_reference(wl))]
+        if net:
+            todo.append(("net_reference", net_reference(wl)))
+        for key, ws in todo:
+            ms_ = weights.handle(zeda, ws)
+            st_total, _ = time_forward(ms_, x, y, args.steps, args.warmup, flush, barrier)
+            Ps, Us, _, _ = ms_.last_counters()
+            ms_.close()
+            refs[key] = {"ms_per_step": st_total / args.steps, "P": Ps, "U": Us, "top_k": ws.K}
+    keys = sorted(refs)
+    red = max_over_ranks([total_ms, e2e_s] + [refs[k]["ms_per_step"] for k in keys], dist, dev)
+    for k, v in zip(keys, red[2:]):
+        refs[k]["ms_per_step"] = v
+    return {"ms_per_step": red[0] / args.steps, "e2e_s": red[1], "P": P, "U": U, "launches": launches,
+            "stage": stage, "refs": refs}
+
+
+def layer_report(wl, name, r, world, steps, peaks, peaks_kind):
+    """The per-workload part of the JSON line from measure_layer's result."""
+    ms = r["ms_per_step"]
+    out = {
+        "value": job_tokens_per_s(world, wl.T, ms), "ms_per_step": ms,
+        "roofline": gemm1_roofline(wl, r["P"], r["U"], float(r["stage"][2]), peaks, peaks_kind, name),
+        "layer_roofline": layer_roofline(wl, r["P"], r["U"], ms, peaks, peaks_kind),
+        "stage_ms": {n: float(v) for n, v in zip(["router", "sort", "gemm1", "gemm2", "combine"], r["stage"])},
+    }
+    for key, ref in r["refs"].items():
+        out[key] = dict(ref, value=world * wl.T / (ref["ms_per_step"] * 1e-3),
+                        speedup_vs_this_reference=ref["ms_per_step"] / ms)
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="decode")
+    ap.add_argument("--workload", default="prefill",
+                    help="prefill (default; carries the decode batch on the same layer as a nested object), decode, "
+                         "tiny, net, glm, sweepNN, prefill_fNN, stack")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-static", action="store_true")
+    ap.add_argument("--no-decode", action="store_true", help="prefill only: skip the nested decode measurement")
     ap.add_argument("--layers", type=int, default=48, help="layers of --workload stack")
     ap.add_argument("--stack-tokens", type=int, default=4096, help="tokens per pass of --workload stack")
     args = ap.parse_args()
@@ -386,116 +565,50 @@ def main():
             dist.destroy_process_group()
         return
     wl = make_workload(args.workload)
-    x_cpu = rank_tokens(wl, rank)
-    m = zeda.from_workload(wl, dev)
-    x = x_cpu.to(dev)
-    y = torch.empty_like(x)
+    weights = DeviceWeights(dev)
     flush = L2Flush(dev)
-
     clocks = ClockSampler(local_rank)
     clocks.start()
-    total_ms, per = time_forward(m, x, y, args.steps, args.warmup, flush, barrier)
-    P, U, zero_slots, launches = m.last_counters()
-
-    # the same steps again with stage events on the stream: duration of the dominant kernel
-    m.set_profiling(True)
-    stage = np.zeros(5)
-    for i in range(args.steps):
-        flush.zero_()
-        m.forward(x, y)
-        stage += np.array(m.stage_ms())
-    stage /= args.steps
-    m.set_profiling(False)
-
-    # end to end through the host-buffer entry point: H2D of x and D2H of y inside the timed region
-    x_pin = x_cpu.pin_memory()
-    y_pin = torch.empty_like(x_pin).pin_memory()
-    for _ in range(args.warmup):
-        flush.zero_()
-        m.forward_host(x_pin, y_pin)
-    barrier()
-    torch.cuda.synchronize()
-    e2e_s = 0.0
-    for i in range(args.steps):
-        flush.zero_()
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        m.forward_host(x_pin, y_pin)
-        e2e_s += time.perf_counter() - t0
-    barrier()
+    headline = args.workload == "prefill"
+    r = measure_layer(zeda, weights, wl, rank_tokens(wl, rank), args, flush, barrier, dist, dev,
+                      static=not args.no_static, net=headline)
     clock_info = clocks.stop()
-
-    # static top-K reference: the same kernels with the zero experts removed (Z = 0)
-    static = None
-    if not args.no_static and wl.Z > 0:
-        ws = inputs.static_reference(wl)
-        ms_ = zeda.from_workload(ws, dev)
-        st_total, _ = time_forward(ms_, x, y, args.steps, args.warmup, flush, barrier)
-        Ps, Us, _, _ = ms_.last_counters()
-        ms_.close()
-        static = {"ms_per_step": st_total / args.steps, "P": Ps, "U": Us}
-
-    # max over ranks
-    total_ms, e2e_s, st_ms = max_over_ranks([total_ms, e2e_s, static["ms_per_step"] if static else 0.0], dist, dev)
-    if static:
-        static["ms_per_step"] = st_ms
+    nested = None
+    if headline and not args.no_decode:
+        # the decode batch on the same layer shape (same expert weights), timed in the same run
+        wd_ = inputs.decode()
+        clocks_d = ClockSampler(local_rank)
+        clocks_d.start()
+        rd = measure_layer(zeda, weights, wd_, rank_tokens(wd_, rank), args, flush, barrier, dist, dev,
+                           e2e=False, static=not args.no_static)
+        nested = (wd_, rd, clocks_d.stop())
 
     if rank == 0:
-        ms_per_step = total_ms / args.steps
-        value = job_tokens_per_s(world, wl.T, ms_per_step)
-        hbm = peaks["hbm_gbs"] * 1e9
-        n_cand = wl.E + wl.Z
-        t_roof, t_flop, t_mem = flops.layer_roofline_seconds(wl.T, wl.d, wl.He, n_cand, P, U,
-                                                             peaks["bf16_tflops"] * 1e12, hbm)
-        # dominant kernel: expert GEMM1 + SwiGLU; algorithmic bytes = gate and up weights of the U
-        # active experts + the x rows it reads + the intermediate it writes
-        names = ["router", "sort", "gemm1", "gemm2", "combine"]
-        g1_bytes = U * 2 * wl.He * wl.d * 2 + wl.T * wl.d * 2 + P * wl.He * 2
-        g1_flops = 4 * P * wl.d * wl.He
-        g1_s = stage[2] * 1e-3
-        # The kernel is timed by stage events inside the step, back to back with the other kernels:
-        # the tensor peak it is held against is the sustained one; the burst figure is given beside it.
-        burst = peaks["bf16_tflops"]
-        sustained = peaks.get("bf16_tflops_sustained", burst)
-        hbm_bound = g1_bytes / hbm >= g1_flops / (sustained * 1e12)
-        if hbm_bound:
-            roof = {"bound": "hbm", "achieved": g1_bytes / g1_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-        else:
-            roof = {"bound": "tensor", "achieved": g1_flops / g1_s / 1e12, "peak": sustained, "unit": "TFLOP/s",
-                    "peak_kind": "sustained (kernel timed inside the step)", "peak_burst": burst,
-                    "frac_of_burst": g1_flops / g1_s / 1e12 / burst}
-        roof["frac"] = roof["achieved"] / roof["peak"]
-        roof.update(traffic=NCU_TRAFFIC_BYTES.get(args.workload), kernel="expert GEMM1 + SwiGLU (expert_gemm_pair_kernel<1,..>)",
-                    peak_source=peaks_kind, algorithmic_bytes=g1_bytes, algorithmic_flops=g1_flops, kernel_ms=stage[2])
-        t_roof_s, t_flop_s, _ = flops.layer_roofline_seconds(wl.T, wl.d, wl.He, n_cand, P, U, sustained * 1e12, hbm)
+        rep = layer_report(wl, args.workload, r, world, args.steps, peaks, peaks_kind)
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "metric": METRIC, "value": rep.pop("value"), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": rep.pop("ms_per_step"), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": workload_config(wl, args.workload, {
-                "P": P, "U": U, "l2": "256 MiB written, then 256 MiB read, between timed steps (outside the event pairs)",
-                "parallelism": "dp%d replicas, no collective" % world}),
+            "config": workload_config(wl, args.workload, r["P"], r["U"], world),
             "clocks": clock_info,
-            "e2e": {"value": world * wl.T * args.steps / e2e_s, "unit": UNIT,
+            "e2e": {"value": world * wl.T * args.steps / r["e2e_s"], "unit": UNIT,
                     "h2d_bytes_per_step": wl.T * wl.d * 2, "d2h_bytes_per_step": wl.T * wl.d * 2,
-                    "ms_per_step": 1e3 * e2e_s / args.steps},
-            "gpu_launches": launches * args.steps,
-            "roofline": roof,
-            "layer_roofline": {"t_roof_us": t_roof * 1e6, "t_flop_us": t_flop * 1e6, "t_hbm_us": t_mem * 1e6,
-                               "frac": t_roof / (ms_per_step * 1e-3), "peak_source": peaks_kind,
-                               "t_flop_us_sustained": t_flop_s * 1e6, "t_roof_us_sustained": t_roof_s * 1e6,
-                               "frac_sustained": t_roof_s / (ms_per_step * 1e-3)},
-            "stage_ms": {n: float(v) for n, v in zip(names, stage)},
+                    "ms_per_step": 1e3 * r["e2e_s"] / args.steps},
+            "gpu_launches": r["launches"] * args.steps,
         }
-        if static:
-            line["static_reference"] = dict(static, value=world * wl.T / (static["ms_per_step"] * 1e-3),
-                                            speedup_vs_static=static["ms_per_step"] / ms_per_step)
+        line.update(rep)
+        if nested:
+            wd_, rd, clk = nested
+            dec = layer_report(wd_, "decode", rd, world, args.steps, peaks, peaks_kind)
+            dec["config"] = workload_config(wd_, "decode", rd["P"], rd["U"], world)
+            dec["clocks"] = clk
+            dec["gpu_launches"] = rd["launches"] * args.steps
+            line["decode"] = dec
         if not args.no_cpu_baseline:
             v, dt, cores, desc = oracle_tokens_per_s(wl, 64, min_seconds=10.0, max_passes=400)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
                                     "seconds": dt}
         print(json.dumps(line))
-    m.close()
     if dist is not None:
         dist.destroy_process_group()
 

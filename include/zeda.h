@@ -80,10 +80,9 @@ typedef struct {
 
 enum {
     ZEDA_FLAG_NONE = 0,
-    ZEDA_FLAG_FORCE_STREAM_EXPERTS = 1, /* always use the weight-streaming expert kernels */
-    ZEDA_FLAG_FORCE_TILE_EXPERTS = 2,   /* always use the single-CTA tcgen05 tile kernels */
     ZEDA_FLAG_NO_DEPENDENT_LAUNCH = 4   /* launch every kernel fully stream-ordered (no programmatic
-                                           dependent launch between the kernels of a call) */
+                                           dependent launch between the kernels of a call); any
+                                           other bit is rejected */
 };
 
 /* Device workspace the handle needs for the given configuration (bytes, multiple of 256);
@@ -189,17 +188,20 @@ zeda_status_t zeda_moe_stage_ms(zeda_moe_t *h, float ms[ZEDA_STAGE_COUNT]);
  * surviving pairs per normal expert, exclusive offsets, permutation ordered by expert then token)
  * on top-K indices the caller already has, and keeps its scratch in a fixed array inside the
  * library instead of a workspace.
- *   topk_idx        dev [T, top_k] int32 candidate ids; ids >= n_real are zero experts (input)
+ *   topk_idx        dev [T, top_k] int32 candidate ids (input); ids >= n_real are zero experts and
+ *                   are dropped, and so is any id < 0 (a padding slot)
  *   expert_counts   dev [n_real] int32          expert_offsets  dev [n_real + 1] int32
  *   perm            dev [T * top_k] int32, first P entries written      n_pairs  dev [1] int32
  * All pointers are required and belong to the CURRENT device.  Limits: T <= ZEDA_STATIC_MAX_TOKENS
  * and T * top_k <= ZEDA_STATIC_MAX_SLOTS, n_real <= 512, top_k <= 16; larger sizes are rejected
  * with ZEDA_ERR_UNSUPPORTED and nothing is launched.  T == 0 returns ZEDA_OK and touches nothing.
- * The scratch array (about 0.4 MB) is part of the library image: every GPU that loads the library
+ * The scratch array (about a third of a megabyte) is part of the library image: every GPU that loads the library
  * holds it until the process exits.  The call makes no cudaMalloc / cudaFree and uses no
  * allocating library routine; it enqueues a small memset and three kernels on `stream`.
  * The first call on each device looks up the array's device address (one cudaGetSymbolAddress,
- * with that device current); make that first call before any stream capture begins.
+ * with that device current); make that first call before any stream capture begins: a first call
+ * on a stream that is being captured is refused with ZEDA_ERR_INVALID_ARG and launches nothing.
+ * Host threads may make their first calls concurrently (the cached address is an atomic).
  * All calls on a device share the one array, which keeps the previous call's contents: the call
  * clears the words that must start at zero itself, but two calls whose work overlaps on the GPU
  * (different streams, or threads) race on it.  Serialise them on one stream. */

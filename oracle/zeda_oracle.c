@@ -18,7 +18,7 @@
  *   - Appendix D: each expert has up, gate and down projections.
  *   - Eq. 4-6: f_i, P_i, L_A, L_GA forward values.
  *
- * Readings where the paper is silent (all listed in the design notes):
+ * Readings taken where the paper is silent:
  *   score function softmax; "normalised routing weight" = softmax restricted to
  *   the K selected logits (mode 0) or the raw softmax entry (mode 1); top-K ties
  *   go to the lower index; expert = down(silu(gate x) * up x) without biases;

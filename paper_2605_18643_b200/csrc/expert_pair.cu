@@ -28,6 +28,8 @@
 // k-step, and that lane's instruction stream is what bounds a narrow tile.  Every mbarrier wait is
 // bounded; on expiry the CTA records an error word, skips the rest of its work, and leaves through
 // the common exit (cluster barrier, TMEM free).
+#include <utility>
+
 #include "tc_common.cuh"
 
 namespace zeda {
@@ -40,7 +42,6 @@ constexpr int kBlockK = 64;                     // bf16 elements per k-step = on
 constexpr int kATileBytes = 128 * kBlockK * 2;  // 16 KB: this CTA's 128 weight rows of one k-step
 constexpr int kRowBytes = kBlockK * 2;          // 128
 constexpr int kAccCols = 256;                   // TMEM columns of one accumulator buffer
-constexpr int kTmemCols = 512;                  // two buffers
 constexpr int kThreads = 256;                   // GEMM2
 constexpr int kThreadsGather = 384;             // GEMM1: + four gather warps
 constexpr int kPatchBytes = 4 * 32 * 32 * 2;    // per epilogue warp: [32 pair rows][32 features] bf16, for 16-byte stores
@@ -82,8 +83,12 @@ __device__ __forceinline__ float swiglu(float g, float u) { return __fdividef(g 
 
 // MODE 1: GEMM1 + SwiGLU -> Hmid[pos, f].   MODE 2: GEMM2 -> O[pos, row].
 // HALF_MAX: most B rows one CTA loads per k-step (the tile's column count is at most 2 * HALF_MAX).
-template <int MODE, int HALF_MAX, int STAGES>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MODE == 1 ? kThreadsGather : kThreads, 1)
+// ACC_BUFS: accumulator buffers in TMEM.  2: one CTA per SM, the epilogue of a tile runs under the MMAs
+// of the CTA's next tile.  1: the CTA takes half of the SM (256 TMEM columns, at most half of the
+// shared memory), two CTAs of different pairs share an SM and fill each other's gaps (epilogues, tiles
+// of few rows that wait on their weight stream).
+template <int MODE, int HALF_MAX, int STAGES, int ACC_BUFS>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MODE == 1 ? kThreadsGather : kThreads, ACC_BUFS == 1 ? 2 : 1)
 expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ RowMaps maps_b,
                         const __nv_bfloat16 *__restrict__ x, int x_ld, const int32_t *__restrict__ counts,
                         const int32_t *__restrict__ offsets, const int32_t *__restrict__ tile_expert,
@@ -91,6 +96,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                         int32_t *__restrict__ meta, int kdim, int out_rows, int m_blocks,
                         __nv_bfloat16 *__restrict__ out, int out_ld) {
     constexpr int kStageBytes = kATileBytes + HALF_MAX * kRowBytes;
+    constexpr int kTmemCols = ACC_BUFS * kAccCols;
     pdl_launch_dependents();
     extern __shared__ __align__(1024) unsigned char pair_smem[];
     __shared__ __align__(8) unsigned long long bars[3 * STAGES + 4];
@@ -225,7 +231,8 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 if (item + stride < n_items) nxt = load_item(item + stride, m_blocks, tile_expert, tile_row0, counts, offsets);
                 const int n_cols = ((it.n + 31) >> 5) << 5;
                 const uint32_t idesc = instr_desc_pair(n_cols);
-                const uint32_t buf = tile_count & 1u, tph = (tile_count >> 1) & 1u;
+                const uint32_t buf = ACC_BUFS == 2 ? (tile_count & 1u) : 0u;
+                const uint32_t tph = (ACC_BUFS == 2 ? (tile_count >> 1) : tile_count) & 1u;
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * buf, tph ^ 1u, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
@@ -332,7 +339,8 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         for (long long item = first; item < n_items && ok; item += stride, ++tile_count) {
             const Item it = nxt;
             if (item + stride < n_items) nxt = load_item(item + stride, m_blocks, tile_expert, tile_row0, counts, offsets);
-            const uint32_t buf = tile_count & 1u, tph = (tile_count >> 1) & 1u;
+            const uint32_t buf = ACC_BUFS == 2 ? (tile_count & 1u) : 0u;
+            const uint32_t tph = (ACC_BUFS == 2 ? (tile_count >> 1) : tile_count) & 1u;
             ok = mbar_wait(bar_tfull + 8 * buf, tph, abort_flag);
             ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp before the aligned TMEM loads
             if (MODE == 1) {
@@ -426,15 +434,30 @@ constexpr int pair_smem_bytes() {
     return STAGES * (kATileBytes + HALF_MAX * kRowBytes) + kPatchBytes + (MODE == 1 ? kXchgBytes : 0) + 1024;
 }
 
-template <int MODE, int HALF_MAX, int STAGES>
-bool set_smem_attr() {
-    return cudaFuncSetAttribute(expert_gemm_pair_kernel<MODE, HALF_MAX, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                pair_smem_bytes<MODE, HALF_MAX, STAGES>()) == cudaSuccess;
-}
+// One configuration of the kernel: its attribute set-up and its launch.
+template <int MODE, int HALF_MAX, int STAGES, int ACC_BUFS>
+struct PairKernel {
+    static constexpr int kSmem = pair_smem_bytes<MODE, HALF_MAX, STAGES>();
+    static bool prepare() {
+        return cudaFuncSetAttribute(expert_gemm_pair_kernel<MODE, HALF_MAX, STAGES, ACC_BUFS>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) == cudaSuccess;
+    }
+    template <typename... Args>
+    static cudaError_t launch(const zeda_moe *h, cudaStream_t s, Args &&...args) {
+        const int ctas_per_sm = ACC_BUFS == 1 ? 2 : 1;
+        const int grid = (h->sm_count / 2) * 2 * ctas_per_sm;
+        return launch_kernel(h->pdl, expert_gemm_pair_kernel<MODE, HALF_MAX, STAGES, ACC_BUFS>, dim3(grid),
+                             dim3(MODE == 1 ? kThreadsGather : kThreads), kSmem, s, std::forward<Args>(args)...);
+    }
+};
 
-// small: at most 64 pair rows per expert (decode batches, T <= 64); big: up to 256 per tile
-constexpr int kSmallHalf = 32, kSmallStages1 = 9, kSmallStages2 = 10;
-constexpr int kBigHalf = 128, kBigStages1 = 6, kBigStages2 = 6;
+// small: at most 64 pair rows per expert (decode batches, T <= 64), a weight stream with many small
+// stages; big: tiles of up to 256 pair rows
+using Gemm1Small = PairKernel<1, 32, 9, 2>;
+using Gemm2Small = PairKernel<2, 32, 10, 2>;
+using Gemm1Big = PairKernel<1, 128, 6, 2>;
+using Gemm2Big = PairKernel<2, 128, 6, 2>;
+constexpr int kSmallTokensMax = 64;
 
 }  // namespace
 
@@ -465,8 +488,7 @@ int init_pair_kernels(zeda_moe *h) {
         const cuuint32_t box[2] = {kBlockK, (cuuint32_t)(128 >> i)};
         ok = ok && encode_bf16_map(&pm->hmid.m[i], h->ws.hmid, 2, dims, strides, box);
     }
-    ok = ok && set_smem_attr<1, kSmallHalf, kSmallStages1>() && set_smem_attr<2, kSmallHalf, kSmallStages2>() &&
-         set_smem_attr<1, kBigHalf, kBigStages1>() && set_smem_attr<2, kBigHalf, kBigStages2>();
+    ok = ok && Gemm1Small::prepare() && Gemm2Small::prepare() && Gemm1Big::prepare() && Gemm2Big::prepare();
     if (!ok) {
         free(pm);
         if (zeda_last_error()[0] == 0) set_error("pair kernel set-up failed: %s", cudaGetErrorString(cudaGetLastError()));
@@ -481,16 +503,11 @@ int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, int T, 
     const Workspace &ws = h->ws;
     const PairMaps *pm = static_cast<const PairMaps *>(h->pmaps);
     const int m_blocks = (c.d_expert + 127) / 128;
-    const int grid = (h->sm_count / 2) * 2;
-    cudaError_t e;
-    if (T <= 2 * kSmallHalf)
-        e = launch_kernel(h->pdl, expert_gemm_pair_kernel<1, kSmallHalf, kSmallStages1>, dim3(grid), dim3(kThreadsGather), pair_smem_bytes<1, kSmallHalf, kSmallStages1>(), s,
-            pm->w_gate_up, pm->hmid, x, c.d_model, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
-            ws.meta, c.d_model, c.d_expert, m_blocks, ws.hmid, c.d_expert);
-    else
-        e = launch_kernel(h->pdl, expert_gemm_pair_kernel<1, kBigHalf, kBigStages1>, dim3(grid), dim3(kThreadsGather), pair_smem_bytes<1, kBigHalf, kBigStages1>(), s,
-            pm->w_gate_up, pm->hmid, x, c.d_model, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
-            ws.meta, c.d_model, c.d_expert, m_blocks, ws.hmid, c.d_expert);
+    auto go = [&](auto k) {
+        return decltype(k)::launch(h, s, pm->w_gate_up, pm->hmid, x, c.d_model, ws.counts, ws.offsets, ws.ptile_expert,
+                                   ws.ptile_row0, ws.pair_token, ws.meta, c.d_model, c.d_expert, m_blocks, ws.hmid, c.d_expert);
+    };
+    const cudaError_t e = T <= kSmallTokensMax ? go(Gemm1Small{}) : go(Gemm1Big{});
     return e == cudaSuccess ? 1 : -1;
 }
 
@@ -499,16 +516,12 @@ int launch_experts_gemm2_pair(const zeda_moe *h, int T, cudaStream_t s) {
     const Workspace &ws = h->ws;
     const PairMaps *pm = static_cast<const PairMaps *>(h->pmaps);
     const int m_blocks = (c.d_model + 255) / 256;
-    const int grid = (h->sm_count / 2) * 2;
-    cudaError_t e;
-    if (T <= 2 * kSmallHalf)
-        e = launch_kernel(h->pdl, expert_gemm_pair_kernel<2, kSmallHalf, kSmallStages2>, dim3(grid), dim3(kThreads), pair_smem_bytes<2, kSmallHalf, kSmallStages2>(), s,
-            pm->w_down, pm->hmid, (const __nv_bfloat16 *)nullptr, 0, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
-            ws.meta, c.d_expert, c.d_model, m_blocks, ws.obuf, c.d_model);
-    else
-        e = launch_kernel(h->pdl, expert_gemm_pair_kernel<2, kBigHalf, kBigStages2>, dim3(grid), dim3(kThreads), pair_smem_bytes<2, kBigHalf, kBigStages2>(), s,
-            pm->w_down, pm->hmid, (const __nv_bfloat16 *)nullptr, 0, ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token,
-            ws.meta, c.d_expert, c.d_model, m_blocks, ws.obuf, c.d_model);
+    auto go = [&](auto k) {
+        return decltype(k)::launch(h, s, pm->w_down, pm->hmid, (const __nv_bfloat16 *)nullptr, 0, ws.counts, ws.offsets,
+                                   ws.ptile_expert, ws.ptile_row0, ws.pair_token, ws.meta, c.d_expert, c.d_model, m_blocks,
+                                   ws.obuf, c.d_model);
+    };
+    const cudaError_t e = T <= kSmallTokensMax ? go(Gemm2Small{}) : go(Gemm2Big{});
     return e == cudaSuccess ? 1 : -1;
 }
 

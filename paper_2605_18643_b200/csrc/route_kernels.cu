@@ -3,6 +3,8 @@
 // (token, normal expert) pairs by expert in a stable order.
 #include <cooperative_groups.h>
 
+#include <atomic>
+
 #include "zeda_internal.h"
 
 namespace zeda {
@@ -137,7 +139,8 @@ __device__ __forceinline__ void topk_gate_token(const float *__restrict__ row, i
     unsigned key[RPL];
 #pragma unroll
     for (int r = 0; r < RPL; ++r) {
-        const unsigned u = __float_as_uint(v[r]);
+        unsigned u = __float_as_uint(v[r]);
+        if (u == 0x80000000u) u = 0u;  // -0 and +0 are equal logits: the lower id decides between them
         key[r] = (r * 32 + lane < n_cand) ? ((u & 0x80000000u) ? ~u : (u | 0x80000000u)) : 0u;
     }
     float my_p = 0.f;
@@ -201,7 +204,7 @@ slot_hist_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real,
     const int s1 = min(T * K, s0 + kSortTokens * K);
     for (int s = s0 + threadIdx.x; s < s1; s += blockDim.x) {
         const int e = topk_idx[s];
-        if (e < n_real) atomicAdd(&hist[e], 1);
+        if ((unsigned)e < (unsigned)n_real) atomicAdd(&hist[e], 1);  // zero experts and ids < 0 are dropped
     }
     __syncthreads();
     for (int e = threadIdx.x; e < n_real; e += blockDim.x) block_hist[(size_t)blockIdx.x * n_real + e] = hist[e];
@@ -235,45 +238,37 @@ __device__ __forceinline__ void stage_ints(int32_t *__restrict__ dst, const int3
 struct ScanShared {
     int32_t cnt[kMaxCand];
     int32_t off[kMaxCand + 1];
-    int32_t chunk[kMaxCand + 1];
-    int32_t tile[kMaxCand + 1];
-    int32_t ptile[kMaxCand + 1];
+    int32_t ptile[kMaxCand + 1];  // exclusive scan of the experts' tile counts
 };
 
-// From per-expert pair counts in sh.cnt: exclusive offsets, P, U, and the work lists of the expert
-// kernels.  Called by every thread of the CTA (blockDim.x >= n_real); contains CTA barriers.
+// From per-expert pair counts in sh.cnt: exclusive offsets, P, U, and the tile list of the expert
+// kernels (experts in id order, each with its tiles of kPairTileM rows in row order; the last tile of
+// an expert may be ragged).  Called by every thread of the CTA (blockDim.x >= 32); contains CTA
+// barriers.
 __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, int total_slots,
                                                    int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
                                                    int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
                                                    const WorkLists &wl, bool write_global = true,
                                                    int list_part = 0, int list_parts = 1) {
     if (threadIdx.x < 32) {
-        // warp 0 scans the three per-expert sequences in steps of 32 with shuffle prefix sums
-        int base_off = 0, base_chunk = 0, base_tile = 0, base_ptile = 0, active = 0, max_rows = 0;
+        // warp 0 scans the per-expert sequences in steps of 32 with shuffle prefix sums
+        int base_off = 0, base_ptile = 0, active = 0, max_rows = 0;
         for (int e0 = 0; e0 < n_real; e0 += 32) {
             const int i = e0 + threadIdx.x;
             const int c = (i < n_real) ? sh.cnt[i] : 0;
-            const int ch = (c + kChunkRows - 1) / kChunkRows;
-            const int tl = (c + kTileM - 1) / kTileM;
             const int pt = (c + kPairTileM - 1) / kPairTileM;
-            int so = c, sc = ch, st = tl, sp = pt;
+            int so = c, sp = pt;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const int a = __shfl_up_sync(kFull, so, o);
-                const int b = __shfl_up_sync(kFull, sc, o);
-                const int g = __shfl_up_sync(kFull, st, o);
                 const int q = __shfl_up_sync(kFull, sp, o);
-                if ((int)threadIdx.x >= o) { so += a; sc += b; st += g; sp += q; }
+                if ((int)threadIdx.x >= o) { so += a; sp += q; }
             }
             if (i < n_real) {
                 sh.off[i] = base_off + so - c;
-                sh.chunk[i] = base_chunk + sc - ch;
-                sh.tile[i] = base_tile + st - tl;
                 sh.ptile[i] = base_ptile + sp - pt;
             }
             base_off += __shfl_sync(kFull, so, 31);
-            base_chunk += __shfl_sync(kFull, sc, 31);
-            base_tile += __shfl_sync(kFull, st, 31);
             base_ptile += __shfl_sync(kFull, sp, 31);
             active += __popc(__ballot_sync(kFull, c > 0));
             int mx = c;
@@ -283,16 +278,12 @@ __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, i
         }
         if (threadIdx.x == 0) {
             sh.off[n_real] = base_off;
-            sh.chunk[n_real] = base_chunk;
-            sh.tile[n_real] = base_tile;
             sh.ptile[n_real] = base_ptile;
         }
         if (threadIdx.x == 0 && write_global) {
             meta[kMetaPairs] = base_off;
             meta[kMetaActive] = active;
             meta[kMetaZeroSlots] = total_slots - base_off;
-            meta[kMetaChunks] = base_chunk;
-            meta[kMetaTiles] = base_tile;
             meta[kMetaPairTiles] = base_ptile;
             meta[kMetaMaxRows] = max_rows;
             if (n_pairs_out) *n_pairs_out = base_off;
@@ -306,25 +297,20 @@ __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, i
         }
         if (threadIdx.x == 0) offsets[n_real] = sh.off[n_real];
     }
-    // Work lists: every CTA that runs this scan holds the same prefix sums, so the CTAs share the
+    // Tile list: every CTA that runs this scan holds the same prefix sums, so the CTAs share the
     // filling (part list_part of list_parts); a CTA outside that sharing passes list_parts = 0.
     if (list_parts <= 0) return;
-    // work lists: entry i belongs to the expert whose first-entry index is the last one <= i
-    auto fill = [&](const int32_t *first, int rows, int32_t *list_expert, int32_t *list_row0) {
-        const int total = first[n_real];
-        for (int i = list_part * blockDim.x + threadIdx.x; i < total; i += list_parts * blockDim.x) {
-            int lo = 0, hi = n_real;  // invariant: first[lo] <= i < first[hi]
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (first[mid] <= i) lo = mid; else hi = mid;
-            }
-            list_expert[i] = lo;
-            list_row0[i] = (i - first[lo]) * rows;
+    // entry i belongs to the expert whose first-entry index is the last one <= i
+    const int total = sh.ptile[n_real];
+    for (int i = list_part * blockDim.x + threadIdx.x; i < total; i += list_parts * blockDim.x) {
+        int lo = 0, hi = n_real;  // invariant: ptile[lo] <= i < ptile[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (sh.ptile[mid] <= i) lo = mid; else hi = mid;
         }
-    };
-    fill(sh.chunk, kChunkRows, wl.chunk_expert, wl.chunk_row0);
-    fill(sh.tile, kTileM, wl.tile_expert, wl.tile_row0);
-    fill(sh.ptile, kPairTileM, wl.ptile_expert, wl.ptile_row0);
+        wl.ptile_expert[i] = lo;
+        wl.ptile_row0[i] = (i - sh.ptile[lo]) * kPairTileM;
+    }
 }
 
 __global__ void __launch_bounds__(512)
@@ -457,7 +443,7 @@ slot_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real
     // count this warp's slots per expert
     for (int s = w0 + lane; s - lane < w1; s += 32) {
         int e = (s < w1) ? topk_idx[s] : -1;
-        if (e >= n_real) e = -1;
+        if ((unsigned)e >= (unsigned)n_real) e = -1;  // zero experts; ids < 0 are dropped the same way
         const unsigned grp = __match_any_sync(kFull, e);
         if (e >= 0 && (grp & lt) == 0) mine[e] += __popc(grp);
         __syncwarp();
@@ -476,7 +462,7 @@ slot_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real
     for (int s = w0 + lane; s - lane < w1; s += 32) {
         int e = (s < w1) ? topk_idx[s] : -1;
         const bool in_range = s < w1;
-        if (e >= n_real) e = -1;
+        if ((unsigned)e >= (unsigned)n_real) e = -1;  // zero experts; ids < 0 are dropped the same way
         const unsigned grp = __match_any_sync(kFull, e);
         int p = -1;
         if (e >= 0) p = mine[e] + __popc(grp & lt);
@@ -527,7 +513,7 @@ slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n
     for (int u = 0; u < kSlotRegs; ++u) {
         const int s = w0 + 32 * u + lane;
         int e = (32 * u < per_warp && s < w1) ? __ldg(topk_idx + s) : -1;
-        e_reg[u] = e >= n_real ? -1 : e;
+        e_reg[u] = (unsigned)e >= (unsigned)n_real ? -1 : e;
     }
     for (int i = threadIdx.x; i < kPlaceWarps * n_real; i += blockDim.x) pos[i] = 0;
     for (int e = threadIdx.x; e < n_real; e += blockDim.x) { base[e] = 0; sh.cnt[e] = 0; }
@@ -714,7 +700,7 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
     const Workspace &ws = h->ws;
     const int nblk = (T + kSortTokens - 1) / kSortTokens;
     int launches = 4;
-    const WorkLists wl = {ws.chunk_expert, ws.chunk_row0, ws.tile_expert, ws.tile_row0, ws.ptile_expert, ws.ptile_row0};
+    const WorkLists wl = {ws.ptile_expert, ws.ptile_row0};
 #define ZEDA_RPL_DISPATCH(CALL)                        \
     do {                                               \
         if (n_cand <= 64) { CALL(2); }                 \
@@ -787,16 +773,12 @@ namespace {
 constexpr int kStaticMaxTokens = ZEDA_STATIC_MAX_TOKENS;
 constexpr int kStaticMaxSlots = ZEDA_STATIC_MAX_SLOTS;
 constexpr int kStaticBlocks = (kStaticMaxTokens + kSortTokens - 1) / kSortTokens;
-constexpr int kStaticLists = kStaticMaxSlots / kChunkRows + kMaxCand + 1;
+constexpr int kStaticLists = kStaticMaxSlots / kPairTileM + kMaxCand + 1;
 
 struct StaticScratch {
     int32_t block_hist[kStaticBlocks * kMaxCand];
     int32_t inv[kStaticMaxSlots];
     int32_t pair_token[kStaticMaxSlots];
-    int32_t chunk_expert[kStaticLists];
-    int32_t chunk_row0[kStaticLists];
-    int32_t tile_expert[kStaticLists];
-    int32_t tile_row0[kStaticLists];
     int32_t ptile_expert[kStaticLists];
     int32_t ptile_row0[kStaticLists];
     int32_t meta[kMetaCount];
@@ -805,7 +787,8 @@ struct StaticScratch {
 static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
 
 constexpr int kMaxDevices = 64;
-StaticScratch *g_static_ptr[kMaxDevices] = {};  // device address of the array, per device
+// device address of the array, per device; atomic so that host threads may race on the first call
+std::atomic<StaticScratch *> g_static_ptr[kMaxDevices] = {};
 
 }  // namespace
 }  // namespace zeda
@@ -829,23 +812,31 @@ extern "C" zeda_status_t zeda_compact_static(const int32_t *topk_idx, int32_t T,
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) { set_error("cudaGetDevice: %s", cudaGetErrorString(e)); return ZEDA_ERR_CUDA; }
     if (dev < 0 || dev >= kMaxDevices) { set_error("device ordinal %d not supported", dev); return ZEDA_ERR_UNSUPPORTED; }
-    if (!g_static_ptr[dev]) {
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    StaticScratch *sc = g_static_ptr[dev].load(std::memory_order_acquire);
+    if (!sc) {
         // One-time set-up for this device: in host code the array's name is only a stand-in, the
-        // kernels need its device address.
+        // kernels need its device address.  The lookup is not a stream operation, so it must not
+        // happen while the stream is being captured.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        e = cudaStreamIsCapturing(s, &cap);
+        if (e != cudaSuccess) { set_error("cudaStreamIsCapturing: %s", cudaGetErrorString(e)); return ZEDA_ERR_CUDA; }
+        if (cap != cudaStreamCaptureStatusNone) {
+            set_error("zeda_compact_static: the first call on a device must come before stream capture begins");
+            return ZEDA_ERR_INVALID_ARG;
+        }
         void *p = nullptr;
         e = cudaGetSymbolAddress(&p, g_static_scratch);
         if (e != cudaSuccess || !p) { set_error("cudaGetSymbolAddress: %s", cudaGetErrorString(e)); return ZEDA_ERR_CUDA; }
-        g_static_ptr[dev] = static_cast<StaticScratch *>(p);
+        sc = static_cast<StaticScratch *>(p);
+        g_static_ptr[dev].store(sc, std::memory_order_release);  // every thread would store the same address
     }
-    StaticScratch *sc = g_static_ptr[dev];
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
     // the array keeps the previous call's contents; the counters start from zero every call
     e = cudaMemsetAsync(sc->meta, 0, sizeof(sc->meta), s);
     if (e != cudaSuccess) { set_error("cudaMemsetAsync: %s", cudaGetErrorString(e)); return ZEDA_ERR_CUDA; }
     const int nblk = (T + kSortTokens - 1) / kSortTokens;
     slot_hist_kernel<<<nblk, 256, sizeof(int32_t) * n_real, s>>>(topk_idx, T, top_k, n_real, sc->block_hist);
-    const WorkLists wl = {sc->chunk_expert, sc->chunk_row0, sc->tile_expert, sc->tile_row0, sc->ptile_expert,
-                          sc->ptile_row0};
+    const WorkLists wl = {sc->ptile_expert, sc->ptile_row0};
     expert_scan_kernel<<<1, 512, 0, s>>>(sc->block_hist, nblk, n_real, T * top_k, expert_counts, expert_offsets,
                                          n_pairs, sc->meta, wl);
     slot_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * kPlaceWarps * n_real, s>>>(

@@ -36,13 +36,13 @@ bool config_ok(const zeda_moe_config_t *c, const char **why) {
     else if ((long long)c->max_tokens * c->top_k >= (1LL << 27)) w = "max_tokens * top_k must be < 2^27";
     else if (c->gate_mode < 0 || c->gate_mode > 2) w = "unknown gate_mode";
     else if (c->expert_kind < 0 || c->expert_kind > 1) w = "unknown expert_kind";
-    else if ((c->flags & ZEDA_FLAG_FORCE_STREAM_EXPERTS) && (c->flags & ZEDA_FLAG_FORCE_TILE_EXPERTS)) w = "contradictory flags";
+    else if (c->flags & ~ZEDA_FLAG_NO_DEPENDENT_LAUNCH) w = "unknown flag";
     if (why) *why = w;
     return w == nullptr;
 }
 
 // Walks the workspace layout; with base == nullptr it only measures.
-size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int *max_chunks, int *max_tiles) {
+size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int *max_tiles) {
     size_t off = 0;
     auto take = [&](size_t bytes) -> void * {
         void *p = base ? base + off : nullptr;
@@ -52,8 +52,7 @@ size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int
     const size_t slots = (size_t)c.max_tokens * c.top_k;
     const size_t n_cand = (size_t)c.n_real + c.n_zero;
     const size_t nblk = (c.max_tokens + kSortTokens - 1) / kSortTokens;
-    const size_t chunks = slots / kChunkRows + c.n_real + 1;
-    const size_t tiles = slots / kTileM + c.n_real + 1;
+    const size_t tiles = slots / kPairTileM + c.n_real + 1;
     const size_t nblk_stats = (c.max_tokens + 63) / 64;
     Workspace w;
     w.topk_idx = (int32_t *)take(slots * 4);
@@ -65,10 +64,6 @@ size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int
     w.counts = (int32_t *)take((size_t)c.n_real * 4);
     w.offsets = (int32_t *)take((size_t)(c.n_real + 1) * 4);
     w.meta = (int32_t *)take(kMetaCount * 4);
-    w.chunk_expert = (int32_t *)take(chunks * 4);
-    w.chunk_row0 = (int32_t *)take(chunks * 4);
-    w.tile_expert = (int32_t *)take(tiles * 4);
-    w.tile_row0 = (int32_t *)take(tiles * 4);
     w.ptile_expert = (int32_t *)take(tiles * 4);
     w.ptile_row0 = (int32_t *)take(tiles * 4);
     w.logits = (float *)take((size_t)router_part_rows(c.max_tokens) * n_cand * 4);
@@ -77,11 +72,9 @@ size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int
     w.hmid = (__nv_bfloat16 *)take((slots + kPairTileM) * c.d_expert * 2);
     w.obuf = (__nv_bfloat16 *)take((slots + kPairTileM) * c.d_model * 2);
     w.router_split = (__nv_bfloat16 *)take((size_t)3 * router_split_pad((int)n_cand) * c.d_model * 2);
-    w.x_sorted = (__nv_bfloat16 *)take((slots + kPairTileM) * c.d_model * 2);
     w.x_stage = (__nv_bfloat16 *)take((size_t)c.max_tokens * c.d_model * 2);
     w.y_stage = (__nv_bfloat16 *)take((size_t)c.max_tokens * c.d_model * 2);
     if (ws) *ws = w;
-    if (max_chunks) *max_chunks = (int)chunks;
     if (max_tiles) *max_tiles = (int)tiles;
     return off;
 }
@@ -137,18 +130,11 @@ zeda_status_t forward_device(zeda_moe_t *h, const __nv_bfloat16 *x, int T, __nv_
     if (r < 0) return cuda_fail("routing launch", cudaGetLastError());
     n += r;
     mark(2);
-    const bool stream = (h->cfg.flags & ZEDA_FLAG_FORCE_STREAM_EXPERTS) != 0;
-    const bool tile = (h->cfg.flags & ZEDA_FLAG_FORCE_TILE_EXPERTS) != 0;
-    if (tile) {
-        r = launch_gather_rows(h, x, T, s);
-        if (r < 0) return cuda_fail("row gather launch", cudaGetLastError());
-        n += r;
-    }
-    r = stream ? launch_experts_gemm1(h, x, T, s) : tile ? launch_experts_gemm1_tile(h, T, s) : launch_experts_gemm1_pair(h, x, T, s);
+    r = launch_experts_gemm1_pair(h, x, T, s);
     if (r < 0) return cuda_fail("expert GEMM1 launch", cudaGetLastError());
     n += r;
     mark(3);
-    r = stream ? launch_experts_gemm2(h, T, s) : tile ? launch_experts_gemm2_tile(h, T, s) : launch_experts_gemm2_pair(h, T, s);
+    r = launch_experts_gemm2_pair(h, T, s);
     if (r < 0) return cuda_fail("expert GEMM2 launch", cudaGetLastError());
     n += r;
     mark(4);
@@ -175,7 +161,7 @@ extern "C" {
 size_t zeda_moe_workspace_bytes(const zeda_moe_config_t *cfg) {
     const char *why = nullptr;
     if (!config_ok(cfg, &why)) { set_error("%s", why); return 0; }
-    return carve(*cfg, nullptr, nullptr, nullptr, nullptr);
+    return carve(*cfg, nullptr, nullptr, nullptr);
 }
 
 zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_w, const float *router_bias,
@@ -195,7 +181,7 @@ zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_
         return ZEDA_ERR_INVALID_ARG;
     }
     if (reinterpret_cast<uintptr_t>(workspace) & 255u) { set_error("workspace must be 256-byte aligned"); return ZEDA_ERR_INVALID_ARG; }
-    const size_t need = carve(*cfg, nullptr, nullptr, nullptr, nullptr);
+    const size_t need = carve(*cfg, nullptr, nullptr, nullptr);
     if (workspace_bytes < need) { set_error("workspace has %zu bytes, %zu needed", workspace_bytes, need); return ZEDA_ERR_WORKSPACE; }
     int ndev = 0;
     cudaError_t e = cudaGetDeviceCount(&ndev);
@@ -218,18 +204,15 @@ zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_
     h->sm_count = prop.multiProcessorCount;
     h->pdl = !(cfg->flags & ZEDA_FLAG_NO_DEPENDENT_LAUNCH);
     h->last_launches = 0;
-    h->tmaps = nullptr;
     h->pmaps = nullptr;
     h->router_maps = nullptr;
     h->profiling = false;
     h->profiled_last = false;
     for (auto &ev : h->ev) ev = nullptr;
-    carve(*cfg, static_cast<unsigned char *>(workspace), &h->ws, &h->max_chunks, &h->max_tiles);
+    carve(*cfg, static_cast<unsigned char *>(workspace), &h->ws, &h->max_tiles);
     if (init_route_kernels(h) < 0) { delete h; return cuda_fail("kernel set-up", cudaGetLastError()); }
-    if (init_tile_kernels(h) < 0) { delete h; return ZEDA_ERR_CUDA; }
-    if (init_pair_kernels(h) < 0) { free(h->tmaps); delete h; return ZEDA_ERR_CUDA; }
+    if (init_pair_kernels(h) < 0) { delete h; return ZEDA_ERR_CUDA; }
     if (init_router_tile(h) < 0) {
-        if (h->tmaps) free(h->tmaps);
         if (h->pmaps) free(h->pmaps);
         delete h;
         return cuda_fail("router set-up", cudaGetLastError());
@@ -399,7 +382,6 @@ zeda_status_t zeda_moe_destroy(zeda_moe_t *h) {
         else if (err != 0) { set_error("a bounded device wait expired (code %d)", err); st = ZEDA_ERR_TIMEOUT; }
     }
     for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
-    if (h->tmaps) free(h->tmaps);
     if (h->pmaps) free(h->pmaps);
     if (h->router_maps) free(h->router_maps);
     delete h;

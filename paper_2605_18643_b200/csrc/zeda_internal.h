@@ -12,20 +12,16 @@ namespace zeda {
 constexpr int kMaxCand = 512;       // N + N_Z limit (16 logits per lane in the top-K warp)
 constexpr int kMaxTopK = 16;
 constexpr int kSortTokens = 128;    // tokens per CTA in the counting sort (histogram / placement)
-constexpr int kChunkRows = 32;      // pair rows per work chunk of the streaming expert kernels
-constexpr int kTileM = 128;         // pair rows per tile of the single-CTA tcgen05 expert kernels
-constexpr int kPairTileM = 256;     // pair rows per tile of the CTA-pair tcgen05 expert kernels
+constexpr int kPairTileM = 256;     // pair rows per tile of the expert kernels (one CTA pair, N <= 256)
 
 // Device-resident counters of one call.
 enum MetaSlot {
     kMetaPairs = 0,      // P
     kMetaActive = 1,     // U
     kMetaZeroSlots = 2,  // slots that landed on zero experts
-    kMetaChunks = 3,     // work chunks for the streaming kernels
-    kMetaTiles = 4,      // M tiles for the tile kernels
     kMetaError = 5,      // sticky error word written by bounded device waits
     kMetaMaxRows = 6,    // largest per-expert pair count
-    kMetaPairTiles = 7,  // tiles for the CTA-pair kernels
+    kMetaPairTiles = 7,  // entries of the expert kernels' tile list
     kMetaCount = 16
 };
 
@@ -39,26 +35,21 @@ struct Workspace {
     int32_t *counts;       // [N]
     int32_t *offsets;      // [N+1]
     int32_t *meta;         // [kMetaCount]
-    int32_t *chunk_expert; // [maxChunks]
-    int32_t *chunk_row0;   // [maxChunks]
-    int32_t *tile_expert;  // [maxTiles]
-    int32_t *tile_row0;    // [maxTiles]
-    int32_t *ptile_expert; // [maxTiles] tiles of kPairTileM rows
-    int32_t *ptile_row0;   // [maxTiles]
+    int32_t *ptile_expert; // [maxTiles] tiles of at most kPairTileM pair rows of one expert
+    int32_t *ptile_row0;   // [maxTiles] first row of the tile within its expert
     float *logits;         // [maxT*(N+N_Z)]
     float *stat_part;      // [nblk_stats * 2 * (N+N_Z)]
     __nv_bfloat16 *hmid;   // [maxT*K, He]
     __nv_bfloat16 *obuf;   // [maxT*K, d]
     __nv_bfloat16 *router_split; // [3][pad128(N+N_Z)][d] bf16 hi/mid/lo pieces of the router rows
-    __nv_bfloat16 *x_sorted; // [maxT*K, d] x rows in pair order (tile path)
     __nv_bfloat16 *x_stage;// [maxT, d]
     __nv_bfloat16 *y_stage;// [maxT, d]
 };
 
-struct WorkLists {  // device-side work lists written by the expert scan
-    int32_t *chunk_expert, *chunk_row0;  // chunks of kChunkRows pair rows
-    int32_t *tile_expert, *tile_row0;    // tiles of kTileM pair rows
-    int32_t *ptile_expert, *ptile_row0;  // tiles of kPairTileM pair rows
+// Device-side tile list written by the expert scan: experts in id order, each with its tiles of at
+// most kPairTileM pair rows in row order.
+struct WorkLists {
+    int32_t *ptile_expert, *ptile_row0;
 };
 
 struct RouteOut {  // where one routing pass writes (user buffers or workspace)
@@ -81,11 +72,9 @@ struct zeda_moe {
     const __nv_bfloat16 *w_down;
     zeda::Workspace ws;
     int sm_count;
-    int max_chunks;
     int max_tiles;
     int last_launches;
-    void *tmaps;  // host-side tensor maps of the tile path (owned)
-    void *pmaps;  // host-side tensor maps of the CTA-pair path (owned)
+    void *pmaps;  // host-side tensor maps of the expert kernels (owned)
     void *router_maps;  // host-side tensor map of the split router weights (owned)
     bool profiling;
     bool profiled_last;
@@ -105,9 +94,6 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
                              int n_parts = 1);
 int launch_stats(const zeda_moe *h, const float *logits, const int32_t *topk_idx, int T, float *f,
                  float *p_mean, float *out, cudaStream_t s);
-int launch_experts_gemm1(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
-int launch_experts_gemm2(const zeda_moe *h, int T, cudaStream_t s);
-int init_tile_kernels(zeda_moe *h);
 int router_split_pad(int n_cand);
 int init_router_tile(zeda_moe *h);
 constexpr int kRouterMaxSplit = 4;
@@ -119,9 +105,6 @@ inline long long router_part_rows(long long max_tokens) {
 }
 int router_split_factor(const zeda_moe *h, int T);
 int launch_router_logits_tile(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, int split, cudaStream_t s);
-int launch_gather_rows(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
-int launch_experts_gemm1_tile(const zeda_moe *h, int T, cudaStream_t s);
-int launch_experts_gemm2_tile(const zeda_moe *h, int T, cudaStream_t s);
 int init_pair_kernels(zeda_moe *h);
 int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
 int launch_experts_gemm2_pair(const zeda_moe *h, int T, cudaStream_t s);

@@ -19,7 +19,7 @@ STAGES = ("router", "sort", "gemm1", "gemm2", "combine")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 GATE_TOPK_NORM, GATE_SOFTMAX_RAW, GATE_RENORM_REAL = 0, 1, 2
 EXPERT_ZERO, EXPERT_COPY = 0, 1
-FLAG_NONE, FLAG_FORCE_STREAM_EXPERTS, FLAG_FORCE_TILE_EXPERTS, FLAG_NO_DEPENDENT_LAUNCH = 0, 1, 2, 4
+FLAG_NONE, FLAG_NO_DEPENDENT_LAUNCH = 0, 4
 
 EXPORTS = (
     "zeda_moe_workspace_bytes", "zeda_moe_create", "zeda_route", "zeda_route_from_logits",

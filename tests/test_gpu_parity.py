@@ -134,7 +134,15 @@ def test_route_from_logits_is_bit_exact_with_ties(zeda):
     l = rng.standard_normal((300, wl.E + wl.Z)).astype(np.float32)
     l[:50] = np.round(l[:50] * 2) / 2          # many exact ties
     l[50] = 0.0
+    # zeros of both signs are equal logits: the lower id wins whatever its sign bit
+    l[51] = np.where(np.arange(wl.E + wl.Z) % 2 == 0, -0.0, 0.0)
+    l[52] = np.where(np.arange(wl.E + wl.Z) % 3 == 0, 0.0, -0.0)
+    l[53] = -1.0
+    l[53, [5, 2, 9]] = [-0.0, 0.0, -0.0]
+    l[54] = np.where(rng.random(wl.E + wl.Z) < 0.5, -0.0, 0.0)
+    assert np.signbit(l[51, 0]) and not np.signbit(l[51, 1])
     idx, w = oracle.route(l, wl.E, wl.Z, wl.K)
+    assert list(idx[51]) == [0, 1] and list(idx[53]) == [2, 5]
     counts, offsets, perm, P = oracle.compact(idx, wl.E)
     o = m.route_from_logits(torch.from_numpy(l).to(dev))
     torch.cuda.synchronize()
@@ -263,12 +271,6 @@ def test_router_with_sliced_reduction_axis(zeda, T, max_tokens):
     m.close()
 
 
-def test_streaming_expert_kernels(zeda):
-    # the weight-streaming expert kernels (register MMAs) stay selectable by flag
-    run_layer(zeda, inputs.tiny(seed=3), flags=1)
-    run_layer(zeda, inputs.tiny(seed=3, T=300), flags=1, token_ids=sample_tokens(300, 40, 2))
-
-
 # ---------------------------------------------------------------------------------- full-size configs
 
 def test_decode_config_full_parity(zeda):
@@ -310,7 +312,9 @@ def test_prefill_config_routing_exact_and_sampled_outputs(zeda):
 def test_sweep_config_sampled(zeda, f):
     wl = inputs.sweep_point(f)
     ids = sample_tokens(wl.T, 64, int(f * 100))
-    err, (P, U, zs) = run_layer(zeda, wl, token_ids=ids, check_routing=False)
+    # routing of all 2048 tokens is compared bit for bit: at this size the router runs on the tensor
+    # cores with its reduction axis in slices
+    err, (P, U, zs) = run_layer(zeda, wl, token_ids=ids)
     assert abs(zs / (wl.T * wl.K) - f) < 0.02
 
 

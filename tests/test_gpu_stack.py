@@ -92,3 +92,62 @@ def test_three_layer_stack_per_layer_parity(zeda):
     for m in mods:
         m.close()
     assert checked == 3
+
+
+def test_qwen_shaped_stack_layers_at_4096_tokens(zeda):
+    # Two consecutive layers of the 48-layer stack workload at its own shape (T = 4096, d = 2048,
+    # 128 + 64 candidates, top-8), with the glue kernel in front of each.  Per layer the oracle is
+    # fed the GPU's own layer input h: routing is compared bit for bit on every token whose
+    # top-(K+1) logits are a margin apart, the compaction on all tokens (the oracle's counting sort
+    # of the GPU's own indices), and y on a token sample.
+    T = 4096
+    dev = torch.device("cuda:0")
+    layers, r0 = inputs.stack_layers(2, T=T)
+    wl0 = layers[0]
+    d, He, E, Z, K = wl0.d, wl0.He, wl0.E, wl0.Z, wl0.K
+    wgu, wd = inputs.expert_weights(E, He, d, 0)
+    wgu_d, wd_d = wgu.to(dev), wd.to(dev)
+    mods = [zeda.ZedaMoE(wl.router_w.to(dev), wl.router_bias.to(dev), wgu_d, wd_d, E, Z, K, T) for wl in layers]
+    r = r0.to(dev).clone()
+    y = None
+    for l, (wl, m) in enumerate(zip(layers, mods)):
+        r_before = r.clone()
+        h = zeda.residual_rmsnorm(r, y)
+        o = m.route(h)
+        y = m.forward(h).clone()
+        torch.cuda.synchronize()
+        r_ref, h_ref = oracle.residual_rmsnorm(_bits(r_before), None if l == 0 else _bits(y_prev))
+        assert np.array_equal(_bits(r), r_ref)
+        hg = h.float().cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(hg - h_ref) <= 1.01 * _ulp_bf16(h_ref))
+        # routing on the GPU's own h
+        lg = oracle.logits(_bits(h), wl.router_w.numpy(), wl.router_bias.numpy())
+        gl = m.router_logits(h).cpu().numpy()
+        assert np.max(np.abs(gl.astype(np.float64) - lg.astype(np.float64))) < 2e-5
+        idx_ref, w_ref = oracle.route(lg, E, Z, K)
+        top = -np.sort(-lg.astype(np.float64), axis=1)[:, : K + 1]
+        clean = np.nonzero(np.min(top[:, :-1] - top[:, 1:], axis=1) >= 1e-3)[0]
+        assert clean.size > 0.85 * T
+        idx_gpu = o["topk_idx"].cpu().numpy()
+        assert np.array_equal(idx_gpu[clean], idx_ref[clean])
+        gw = o["topk_w"].cpu().numpy().astype(np.float64)
+        assert np.allclose(gw[clean], w_ref[clean], rtol=1e-5, atol=1e-30)
+        counts, offsets, perm, P = oracle.compact(idx_gpu, E)
+        assert int(o["n_pairs"].item()) == P
+        assert np.array_equal(o["counts"].cpu().numpy(), counts)
+        assert np.array_equal(o["offsets"].cpu().numpy(), offsets)
+        assert np.array_equal(o["perm"].cpu().numpy()[:P], perm)
+        zero_share = 1.0 - P / (T * K)
+        assert 0.2 < zero_share < 0.8
+        # outputs on a sample of the clean tokens
+        ids = clean[:: max(1, clean.size // 48)].astype(np.int32)
+        y_ref, idx_o, _ = oracle.forward(_bits(h), wl.router_w.numpy(), wl.router_bias.numpy(), inputs.bits(wgu),
+                                         inputs.bits(wd), E, Z, K, token_ids=ids)
+        assert np.array_equal(idx_o, idx_gpu[ids])
+        yg = y[torch.as_tensor(ids, device=dev, dtype=torch.long)].float().cpu().numpy().astype(np.float64)
+        den = np.linalg.norm(y_ref)
+        assert den > 0 and np.linalg.norm(yg - y_ref) / den <= REL_L2
+        assert np.max(np.abs(yg - y_ref)) <= MAX_ABS_RMS * np.sqrt(np.mean(y_ref ** 2))
+        y_prev = y
+    for m in mods:
+        m.close()

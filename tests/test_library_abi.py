@@ -53,7 +53,7 @@ def test_workspace_size_and_config_checks(zeda):
                 zeda.Config(2048, 768, 500, 64, 8, 64, 0, 0, 0, 0),      # too many candidates
                 zeda.Config(2048, 768, 128, 64, 8, 0, 0, 0, 0, 0),       # max_tokens
                 zeda.Config(2048, 768, 128, 64, 8, 64, 7, 0, 0, 0),      # gate mode
-                zeda.Config(2048, 768, 128, 64, 8, 64, 0, 0, 0, 3)):     # contradictory flags
+                zeda.Config(2048, 768, 128, 64, 8, 64, 0, 0, 0, 3)):     # unknown flag bits
         assert zeda.workspace_bytes(bad) == 0
         assert zeda.last_error() != ""
 
