@@ -75,6 +75,59 @@ __device__ __forceinline__ Item load_item(long long item, int m_blocks, const in
     return it;
 }
 
+// ---- work items handed out at run time --------------------------------------------------------
+// The clusters do not own fixed shares of the item list: each takes the next unclaimed item from
+// a device counter whenever its weight producer starts on the item before (an atomic add by one
+// scheduler warp of the leader CTA), so that a cluster that drew cheap items simply draws more of
+// them.  The scheduler packs the item's description into one 64-bit word and stores it into slot
+// (sequence number mod kItemSlots) of a small queue in BOTH CTAs' shared memory; every role reads
+// the sequence of items from its own CTA's queue, polling the slot until its tag matches.
+//   bits 63..51 tag = sequence number mod 8191, plus 1 (never 0: an unwritten slot matches nothing)
+//   bit  50     end of the list          49..41 expert       40..35 weight-row block
+//   34..27      pair rows in the tile - 1                    26..0  first pair position
+// A slot is overwritten kItemSlots items later.  The scheduler runs at most one item ahead of the
+// weight producer, the producer at most STAGES k-steps (at most that many items) ahead of the MMA
+// warp, the MMA warp at most two tiles ahead of the slowest epilogue warp of either CTA (it needs
+// every epilogue warp's arrival to reuse an accumulator): with STAGES <= 10 no reader is more than
+// 15 items behind the scheduler, and kItemSlots = 32.
+constexpr int kItemSlots = 32;
+constexpr int kSchedAhead = 1;  // items the scheduler may run ahead of the weight producer
+
+__device__ __forceinline__ unsigned long long pack_item(uint32_t seq, bool end, const Item &it) {
+    return ((unsigned long long)(seq % 8191u + 1u) << 51) | ((unsigned long long)(end ? 1 : 0) << 50) |
+           ((unsigned long long)(uint32_t)it.e << 41) | ((unsigned long long)(uint32_t)it.mb << 35) |
+           ((unsigned long long)(uint32_t)(it.n - 1) << 27) | (unsigned long long)(uint32_t)it.pos0;
+}
+
+// The item with sequence number seq from this CTA's queue; called by all 32 lanes of a converged warp
+// (lane 0 polls, the word is broadcast).  Returns 1 with the item, 0 at the end of the list, -1 if the
+// entry did not arrive within the wait limit or another role of this CTA gave up.
+__device__ __forceinline__ int next_item(const volatile unsigned long long *queue, uint32_t seq, Item &it,
+                                         volatile int *abort_flag) {
+    const unsigned long long want = seq % 8191u + 1u;
+    unsigned long long v = 0ull;
+    int status = 1;
+    if ((threadIdx.x & 31) == 0) {
+        v = queue[seq % kItemSlots];
+        if ((v >> 51) != want) {
+            const long long t0 = clock64();
+            int spins = 0;
+            while (((v = queue[seq % kItemSlots]) >> 51) != want) {
+                if ((++spins & 63) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) { status = -1; break; }
+            }
+        }
+    }
+    status = __shfl_sync(0xffffffffu, status, 0);
+    if (status < 0) return -1;
+    v = __shfl_sync(0xffffffffu, v, 0);
+    if ((v >> 50) & 1ull) return 0;
+    it.e = (int)((v >> 41) & 0x1ffu);
+    it.mb = (int)((v >> 35) & 0x3fu);
+    it.n = (int)((v >> 27) & 0xffu) + 1;
+    it.pos0 = (int)(v & 0x7ffffffu);
+    return 1;
+}
+
 __device__ __forceinline__ void named_sync(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
@@ -95,6 +148,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                         const int32_t *__restrict__ tile_row0, const int32_t *__restrict__ pair_token,
                         int32_t *__restrict__ meta, int kdim, int out_rows, int m_blocks,
                         __nv_bfloat16 *__restrict__ out, int out_ld) {
+    static_assert(STAGES <= 10, "the item queue's depth assumes at most 10 ring stages");
     constexpr int kStageBytes = kATileBytes + HALF_MAX * kRowBytes;
     constexpr int kTmemCols = ACC_BUFS * kAccCols;
     pdl_launch_dependents();
@@ -103,6 +157,8 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ int s_ok[4];
+    __shared__ __align__(8) unsigned long long s_items[kItemSlots];  // this CTA's copy of the item queue
+    __shared__ int s_prod_seq;                                       // item the weight producer is on (leader CTA)
 
     // 1024-byte alignment of the operand ring (the swizzle pattern is a function of the address)
     const uint32_t ring = (smem_u32(pair_smem) + 1023u) & ~1023u;
@@ -118,8 +174,10 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     const uint32_t rank = cluster_ctarank();
     const bool leader = rank == 0;
 
+    if (threadIdx.x < kItemSlots) s_items[threadIdx.x] = 0ull;
     if (threadIdx.x == 0) {
         s_abort = 0;
+        s_prod_seq = -1;
         // full: the TMA producer's expect_tx arrival (+ GEMM1: the gather relay of each CTA)
         for (int i = 0; i < STAGES; ++i) {
             mbar_init(bar_full + 8 * i, MODE == 1 ? 3 : 1);
@@ -139,9 +197,8 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     volatile int *abort_flag = &s_abort;
     pdl_wait();  // everything above is local set-up; the routing results and activations are read below
 
-    const long long n_items = (long long)meta[kMetaPairTiles] * m_blocks;
     const int k_steps = kdim / kBlockK;
-    const long long first = blockIdx.x >> 1, stride = gridDim.x >> 1;
+    const volatile unsigned long long *queue = s_items;
     const uint32_t full0 = mapa(bar_full, 0);      // the leader's full barriers, as seen from either CTA
     const uint32_t tempty0 = mapa(bar_tempty, 0);  // the leader's accumulator-free barriers
 
@@ -150,11 +207,11 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         {
             uint32_t it_count = 0;
             bool ok = true;
-            Item nxt = {0, 0, 0, 0};  // the next item's description is fetched while this one is processed
-            if (first < n_items) nxt = load_item(first, m_blocks, tile_expert, tile_row0, counts, offsets);
-            for (long long item = first; item < n_items && ok; item += stride) {
-                const Item it = nxt;
-                if (item + stride < n_items) nxt = load_item(item + stride, m_blocks, tile_expert, tile_row0, counts, offsets);
+            for (uint32_t seq = 0; ok; ++seq) {
+                Item it;
+                const int got = next_item(queue, seq, it, abort_flag);
+                if (got <= 0) { ok = got == 0; break; }
+                if (lane == 0) *reinterpret_cast<volatile int *>(&s_prod_seq) = (int)seq;  // read by the scheduler warp
                 const int half = ((it.n + 31) >> 5) << 4;  // B rows of this CTA; the tile has 2 * half columns
                 const uint32_t bytes = 2u * (uint32_t)(kATileBytes + (MODE == 2 ? half * kRowBytes : 0));
                 for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
@@ -184,11 +241,10 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         {
             uint32_t it_count = 0;
             bool ok = true;
-            Item nxt = {0, 0, 0, 0};  // the next item's description is fetched while this one is processed
-            if (first < n_items) nxt = load_item(first, m_blocks, tile_expert, tile_row0, counts, offsets);
-            for (long long item = first; item < n_items && ok; item += stride) {
-                const Item it = nxt;
-                if (item + stride < n_items) nxt = load_item(item + stride, m_blocks, tile_expert, tile_row0, counts, offsets);
+            for (uint32_t seq = 0; ok; ++seq) {
+                Item it;
+                const int got = next_item(queue, seq, it, abort_flag);
+                if (got <= 0) { ok = got == 0; break; }
                 const int half = ((it.n + 31) >> 5) << 4;
                 const int brow0 = (int)rank * half;  // first tile column / pair row this CTA loads
                 for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
@@ -224,11 +280,10 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             // descriptors of stage 0; stage s is (s * kStageBytes) >> 4 further in the address field
             const uint64_t a0 = smem_desc_sw128(ring), b0 = smem_desc_sw128(ring + kATileBytes);
             bool ok = true;
-            Item nxt = {0, 0, 0, 0};  // the next item's description is fetched while this one is processed
-            if (first < n_items) nxt = load_item(first, m_blocks, tile_expert, tile_row0, counts, offsets);
-            for (long long item = first; item < n_items && ok; item += stride, ++tile_count) {
-                const Item it = nxt;
-                if (item + stride < n_items) nxt = load_item(item + stride, m_blocks, tile_expert, tile_row0, counts, offsets);
+            for (uint32_t seq = 0; ok; ++seq, ++tile_count) {
+                Item it;
+                const int got = next_item(queue, seq, it, abort_flag);
+                if (got <= 0) { ok = got == 0; break; }
                 const int n_cols = ((it.n + 31) >> 5) << 5;
                 const uint32_t idesc = instr_desc_pair(n_cols);
                 const uint32_t buf = ACC_BUFS == 2 ? (tile_count & 1u) : 0u;
@@ -268,7 +323,10 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         {
             uint32_t it_count = 0;
             bool ok = true;
-            for (long long item = first; item < n_items && ok; item += stride) {
+            for (uint32_t seq = 0; ok; ++seq) {
+                Item it;
+                const int got = next_item(queue, seq, it, abort_flag);
+                if (got <= 0) { ok = got == 0; break; }
                 for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
                     const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
                     ok = __all_sync(0xffffffffu, mbar_wait(bar_gfull + 8 * s, ph, abort_flag));
@@ -279,6 +337,43 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             }
             if (!ok && lane == 0) {
                 if (!*abort_flag) atomicExch(&meta[kMetaError], 15);
+                s_abort = 1;
+            }
+        }
+    } else if (warp == (MODE == 1 ? 3 : 2)) {
+        // ------------------------------------------------------------------ item scheduler (leader CTA)
+        if (leader) {
+            const long long n_items = (long long)meta[kMetaPairTiles] * m_blocks;
+            int32_t *counter = meta + (MODE == 1 ? kMetaNextItem1 : kMetaNextItem2);
+            const uint32_t peer_queue = mapa(smem_u32(s_items), 1);
+            const volatile int *prod_seq = &s_prod_seq;
+            bool ok = true;
+            for (uint32_t seq = 0; ok; ++seq) {
+                // at most kSchedAhead items ahead of the one the weight producer is loading
+                if (lane == 0 && (int)seq > *prod_seq + kSchedAhead) {
+                    const long long t0 = clock64();
+                    int spins = 0;
+                    while ((int)seq > *prod_seq + kSchedAhead) {
+                        __nanosleep(64);
+                        if ((++spins & 63) == 0 && (*abort_flag || clock64() - t0 > kWaitLimitCycles)) { ok = false; break; }
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                bool end = false;
+                if (lane == 0) {
+                    const long long item = atomicAdd(counter, 1);
+                    Item it = {0, 0, 1, 0};
+                    end = item >= n_items;
+                    if (!end) it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
+                    const unsigned long long rec = pack_item(seq, end, it);
+                    asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(peer_queue + 8 * (seq % kItemSlots)), "l"(rec) : "memory");
+                    *reinterpret_cast<volatile unsigned long long *>(&s_items[seq % kItemSlots]) = rec;
+                }
+                if (__shfl_sync(0xffffffffu, end, 0)) break;
+            }
+            if (!ok && lane == 0) {
+                if (!*abort_flag) atomicExch(&meta[kMetaError], 17);
                 s_abort = 1;
             }
         }
@@ -293,11 +388,10 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         const uint32_t dst_off = (uint32_t)(rsub * kRowBytes + ((chunk ^ (rsub & 7)) << 4));
         uint32_t it_count = 0;
         bool ok = true;
-        Item nxt = {0, 0, 0, 0};  // the next item's description is fetched while this one is processed
-        if (first < n_items) nxt = load_item(first, m_blocks, tile_expert, tile_row0, counts, offsets);
-        for (long long item = first; item < n_items && ok; item += stride) {
-            const Item it = nxt;
-            if (item + stride < n_items) nxt = load_item(item + stride, m_blocks, tile_expert, tile_row0, counts, offsets);
+        for (uint32_t seq = 0; ok; ++seq) {
+            Item it;
+            const int got = next_item(queue, seq, it, abort_flag);
+            if (got <= 0) { ok = got == 0; break; }
             const int half = ((it.n + 31) >> 5) << 4;
             const int brow0 = (int)rank * half;
             const __nv_bfloat16 *src[HALF_MAX / 16];
@@ -334,23 +428,21 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         const int prow = lane >> 2, pch = lane & 3;  // 16-byte piece this lane stores: rows prow + 8 i, features 8 pch ..
         uint32_t tile_count = 0;
         bool ok = true;
-        Item nxt = {0, 0, 0, 0};  // the next item's description is fetched while this one is processed
-        if (first < n_items) nxt = load_item(first, m_blocks, tile_expert, tile_row0, counts, offsets);
-        for (long long item = first; item < n_items && ok; item += stride, ++tile_count) {
-            const Item it = nxt;
-            if (item + stride < n_items) nxt = load_item(item + stride, m_blocks, tile_expert, tile_row0, counts, offsets);
+        for (uint32_t seq = 0; ok; ++seq, ++tile_count) {
+            Item it;
+            int status = next_item(queue, seq, it, abort_flag);  // 1 item, 0 end of the list, -1 gave up
             const uint32_t buf = ACC_BUFS == 2 ? (tile_count & 1u) : 0u;
             const uint32_t tph = (ACC_BUFS == 2 ? (tile_count >> 1) : tile_count) & 1u;
-            ok = mbar_wait(bar_tfull + 8 * buf, tph, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);  // also reconverges the warp before the aligned TMEM loads
+            if (status > 0 && !mbar_wait(bar_tfull + 8 * buf, tph, abort_flag)) status = -1;
+            status = __reduce_min_sync(0xffffffffu, status);  // also reconverges the warp before the aligned TMEM loads
             if (MODE == 1) {
-                // the two warps of a pair meet at named barriers below: they must take the same branch
-                if (lane == 0) s_ok[q] = ok ? 1 : 0;
+                // the two warps of a pair meet at named barriers below: they must leave the loop together
+                if (lane == 0) s_ok[q] = status;
                 named_sync(1 + wp, 64);
-                ok = s_ok[wp] && s_ok[wp + 2];
+                status = min(s_ok[wp], s_ok[wp + 2]);
                 named_sync(1 + wp, 64);
             }
-            if (!ok) break;
+            if (status <= 0) { ok = status == 0; break; }
             tc_fence_after();
             const uint32_t t0 = tmem_base + ((uint32_t)(32 * q) << 16) + buf * kAccCols;
             if (MODE == 1) {

@@ -286,6 +286,8 @@ __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, i
             meta[kMetaZeroSlots] = total_slots - base_off;
             meta[kMetaPairTiles] = base_ptile;
             meta[kMetaMaxRows] = max_rows;
+            meta[kMetaNextItem1] = 0;
+            meta[kMetaNextItem2] = 0;
             if (n_pairs_out) *n_pairs_out = base_off;
         }
     }

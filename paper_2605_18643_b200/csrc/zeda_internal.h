@@ -22,6 +22,8 @@ enum MetaSlot {
     kMetaError = 5,      // sticky error word written by bounded device waits
     kMetaMaxRows = 6,    // largest per-expert pair count
     kMetaPairTiles = 7,  // entries of the expert kernels' tile list
+    kMetaNextItem1 = 8,  // next unclaimed work item of the GEMM1 kernel (reset by the routing pass)
+    kMetaNextItem2 = 9,  // the same for GEMM2
     kMetaCount = 16
 };
 
