@@ -43,7 +43,8 @@ typedef enum {
     ZEDA_ERR_UNSUPPORTED = -2, /* a shape the kernels do not cover (see zeda_moe_config_t) */
     ZEDA_ERR_WORKSPACE = -3,   /* workspace smaller than zeda_moe_workspace_bytes() */
     ZEDA_ERR_CUDA = -4,        /* a CUDA runtime call failed; text in zeda_last_error() */
-    ZEDA_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (reported by a later call) */
+    ZEDA_ERR_TIMEOUT = -5      /* a bounded device-side wait expired or a device-side check failed (reported
+                                  by a later call) */
 } zeda_status_t;
 
 /* How the routing weight g~ of a selected slot is formed from p = softmax(logits over N+N_Z).
@@ -76,6 +77,13 @@ typedef struct {
     int32_t expert_kind; /* zeda_expert_kind_t */
     int32_t device;      /* CUDA device ordinal */
     int32_t flags;       /* ZEDA_FLAG_* */
+    /* Expert parallelism (zeda_ep_* calls below).  ep_size = 0: a plain handle that holds all N
+     * experts.  ep_size = G >= 1: this handle is rank ep_rank of a group of G; it routes over all
+     * N + N_Z candidates but holds only the weights of experts [ep_rank * N/G, (ep_rank+1) * N/G)
+     * (N must be a multiple of G, G <= 64) and can take in up to max_recv_pairs pair rows per call. */
+    int32_t ep_size;
+    int32_t ep_rank;
+    int32_t max_recv_pairs;
 } zeda_moe_config_t;
 
 enum {
@@ -161,6 +169,13 @@ zeda_status_t zeda_residual_rmsnorm(void *r, const void *y, void *h, int32_t T, 
 zeda_status_t zeda_moe_stats(zeda_moe_t *h, const void *x, int32_t T, float *f, float *p_mean,
                              float *out, void *stream);
 
+/* Per-token zero-expert ratio of the most recent routing on this handle (zeda_route, zeda_moe_forward,
+ * zeda_moe_stats or zeda_ep_dispatch): r_ze[t] = (slots of token t that selected a zero expert) / K
+ * (Section 2.2 defines r_ZE; Section 4.1 studies how it varies from token to token).
+ *   T     must be the token count of that routing call      r_ze  dev [T] fp32
+ * Reads the routing kept in the workspace; computes nothing else. */
+zeda_status_t zeda_moe_token_zero_share(zeda_moe_t *h, int32_t T, float *r_ze, void *stream);
+
 /* Counters of the last forward call, read back after synchronising the stream (blocking):
  * out[0] = P (surviving pairs), out[1] = U (normal experts with at least one pair),
  * out[2] = zero-expert slots, out[3] = kernels launched by that call. */
@@ -210,6 +225,44 @@ zeda_status_t zeda_moe_stage_ms(zeda_moe_t *h, float ms[ZEDA_STAGE_COUNT]);
 zeda_status_t zeda_compact_static(const int32_t *topk_idx, int32_t T, int32_t top_k, int32_t n_real,
                                   int32_t *expert_counts, int32_t *expert_offsets, int32_t *perm,
                                   int32_t *n_pairs, void *stream);
+
+/* Expert-parallel forward: the experts are partitioned over G ranks (one handle each), the tokens
+ * stay data-parallel.  Zero-expert slots are dropped BEFORE anything is exchanged, so they cost no
+ * link bytes either (the paper's Appendix A, limitations, points at expert-parallel dispatch in the
+ * DeepEP style as future work; the arithmetic is still Eq. 1).  The library does the device work
+ * of one rank; the caller moves the rows between ranks (an all-to-all with per-rank row counts,
+ * NCCL or any other transport) between the three calls:
+ *
+ *   zeda_ep_dispatch  routes this rank's T tokens (as zeda_route; the routing stays in the handle
+ *                     for the combine) and packs the x rows of the surviving pairs, in the order
+ *                     (expert ascending, token ascending), into send_rows.  Experts are owned in
+ *                     contiguous blocks, so the rows for rank r are the contiguous range that
+ *                     follows the rows for ranks < r.
+ *       x             dev [T, d_model] bf16
+ *       send_rows     dev [T*K, d_model] bf16, first P rows written
+ *       send_counts   dev [G] int32: rows for each destination rank (sum = P)
+ *       expert_counts dev [N] int32: pairs per expert; rank r needs entries [r*N/G, (r+1)*N/G)
+ *   (exchange: every rank sends block r of send_rows and of expert_counts to rank r)
+ *   zeda_ep_experts   runs this rank's experts on the rows received from the group.
+ *       recv_rows     dev [n_rows, d_model] bf16: the blocks received from source ranks 0..G-1 in
+ *                     that order, each in its sender's (expert, token) order
+ *       recv_counts   dev [G, N/G] int32: recv_counts[s][j] = rows from source s for local expert j
+ *       n_rows        sum of recv_counts (host value, <= max_recv_pairs); a mismatch with the
+ *                     device-side sum is recorded like an expired wait (ZEDA_ERR_TIMEOUT later)
+ *       out_rows      dev [n_rows, d_model] bf16: E_i(row), in the order of recv_rows
+ *   (exchange back: block s of out_rows returns to rank s)
+ *   zeda_ep_combine   Eq. 1 on the returned rows, which are in the order of send_rows.
+ *       x             the same activations as in zeda_ep_dispatch (read by copy experts only)
+ *       back_rows     dev [P, d_model] bf16        y  dev [T, d_model] bf16
+ * All three only enqueue kernels on `stream`.  A handle with ep_size >= 1 serves these calls, the
+ * routing calls and zeda_moe_stats, not zeda_moe_forward (its pair buffers are sized by
+ * max_recv_pairs); with G = 1 the three calls in a row, without an exchange, are the plain layer. */
+zeda_status_t zeda_ep_dispatch(zeda_moe_t *h, const void *x, int32_t T, void *send_rows,
+                               int32_t *send_counts, int32_t *expert_counts, void *stream);
+zeda_status_t zeda_ep_experts(zeda_moe_t *h, const void *recv_rows, const int32_t *recv_counts,
+                              int32_t n_rows, void *out_rows, void *stream);
+zeda_status_t zeda_ep_combine(zeda_moe_t *h, const void *x, const void *back_rows, int32_t T, void *y,
+                              void *stream);
 
 /* Failure reporting.  Every device-side wait in the tensor-core kernels is bounded; a wait that
  * expires makes its CTA record an error word in the workspace, skip its remaining work and leave

@@ -157,6 +157,15 @@ def stats(logits_f32, topk_idx, n_real, n_zero, alpha=1.0, group_w=1.0):
     return {"f": f, "P": pm, "r_ze": float(out[0]), "L_A": float(out[1]), "L_GA": float(out[2])}
 
 
+def token_zero_share(topk_idx, n_real):
+    """Per-token share of the K slots on zero experts, fp64 [T]."""
+    idx = np.ascontiguousarray(topk_idx, dtype=np.int32)
+    T, K = idx.shape
+    out = np.empty(T, dtype=np.float64)
+    _load().zeda_oracle_token_zero_share(_p(idx), ctypes.c_int(T), ctypes.c_int(n_real), ctypes.c_int(K), _p(out))
+    return out
+
+
 def _bf16_to_f64(bits):
     return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 

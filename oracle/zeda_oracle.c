@@ -262,3 +262,15 @@ void zeda_oracle_stats(const float *logits, const int32_t *topk_idx, int T, int 
     if (n_zero > 0) ga += fZ * pZ / (n_zero * group_w);
     out[2] = alpha * (n_real + n_zero * group_w) / K * ga;
 }
+
+/* Per-token zero-expert ratio: the share of token t's K slots that landed on zero experts
+ * (Section 2.2 defines r_ZE as the fraction of activated experts that are zero experts; Section 4.1
+ * looks at it token by token). */
+void zeda_oracle_token_zero_share(const int32_t *topk_idx, int T, int n_real, int K, double *out) {
+    for (int t = 0; t < T; ++t) {
+        int zero = 0;
+        for (int k = 0; k < K; ++k)
+            if (topk_idx[(size_t)t * K + k] >= n_real) zero++;
+        out[t] = (double)zero / (double)K;
+    }
+}

@@ -75,13 +75,19 @@ combine_kernel(const __nv_bfloat16 *__restrict__ obuf, const int32_t *__restrict
 }  // namespace
 
 int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s) {
+    return launch_combine_rows(h, h->ws.obuf, x, T, y, s);
+}
+
+// rows: the expert outputs of the call's surviving pairs in (expert, token) order
+int launch_combine_rows(const zeda_moe *h, const __nv_bfloat16 *rows, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y,
+                        cudaStream_t s) {
     const zeda_moe_config_t &c = h->cfg;
     // small batches spread a row over several CTAs so that the grid still covers the SMs
     const int chunks = c.d_model / 8;
     int gy = 1;
     while (T * gy < 4 * h->sm_count && gy * kCombineThreads < chunks) gy *= 2;
-    const cudaError_t e = launch_kernel(h->pdl, combine_kernel, dim3(T, gy), dim3(kCombineThreads), 0, s, h->ws.obuf, h->ws.inv,
-                                        h->ws.topk_w, x, c.top_k, c.d_model, (int)(c.expert_kind == ZEDA_EXPERT_COPY), y);
+    const cudaError_t e = launch_kernel(h->pdl, combine_kernel, dim3(T, gy), dim3(kCombineThreads), 0, s, rows, (const int32_t *)h->ws.inv,
+                                        (const float *)h->ws.topk_w, x, c.top_k, c.d_model, (int)(c.expert_kind == ZEDA_EXPERT_COPY), y);
     return e == cudaSuccess ? 1 : -1;
 }
 

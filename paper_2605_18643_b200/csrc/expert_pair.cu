@@ -549,7 +549,14 @@ using Gemm1Small = PairKernel<1, 32, 9, 2>;
 using Gemm2Small = PairKernel<2, 32, 10, 2>;
 using Gemm1Big = PairKernel<1, 128, 6, 2>;
 using Gemm2Big = PairKernel<2, 128, 6, 2>;
-constexpr int kSmallTokensMax = 64;
+constexpr int kSmallRowsMax = 64;
+
+// The small geometry holds at most kSmallRowsMax pair rows of one expert.  Without expert parallelism
+// an expert has at most one pair per token of the call; with it, any number of the received rows.
+bool small_geometry(const zeda_moe *h, const ExpertWork &w) {
+    const int per_expert_bound = h->cfg.ep_size >= 1 ? w.rows_bound : w.rows_bound / h->cfg.top_k;
+    return per_expert_bound <= kSmallRowsMax;
+}
 
 }  // namespace
 
@@ -557,8 +564,8 @@ int init_pair_kernels(zeda_moe *h) {
     const zeda_moe_config_t &c = h->cfg;
     PairMaps *pm = static_cast<PairMaps *>(aligned_alloc(64, sizeof(PairMaps)));
     if (!pm) { set_error("out of host memory"); return -1; }
-    const cuuint64_t E = c.n_real, d = c.d_model, He = c.d_expert;
-    const cuuint64_t rows = (cuuint64_t)c.max_tokens * c.top_k + kPairTileM;
+    const cuuint64_t E = h->n_local, d = c.d_model, He = c.d_expert;
+    const cuuint64_t rows = (cuuint64_t)h->pair_rows + kPairTileM;
     bool ok = true;
     {
         // a 5-D view of [N][2 He][d] that lets one box fetch 64 gate rows and the matching 64 up rows:
@@ -590,30 +597,31 @@ int init_pair_kernels(zeda_moe *h) {
     return 0;
 }
 
-int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s) {
+int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, const ExpertWork &w, cudaStream_t s) {
     const zeda_moe_config_t &c = h->cfg;
     const Workspace &ws = h->ws;
     const PairMaps *pm = static_cast<const PairMaps *>(h->pmaps);
     const int m_blocks = (c.d_expert + 127) / 128;
     auto go = [&](auto k) {
-        return decltype(k)::launch(h, s, pm->w_gate_up, pm->hmid, x, c.d_model, ws.counts, ws.offsets, ws.ptile_expert,
-                                   ws.ptile_row0, ws.pair_token, ws.meta, c.d_model, c.d_expert, m_blocks, ws.hmid, c.d_expert);
+        return decltype(k)::launch(h, s, pm->w_gate_up, pm->hmid, x, c.d_model, w.counts, w.offsets, w.tile_expert,
+                                   w.tile_row0, w.pair_row, ws.meta, c.d_model, c.d_expert, m_blocks, ws.hmid, c.d_expert);
     };
-    const cudaError_t e = T <= kSmallTokensMax ? go(Gemm1Small{}) : go(Gemm1Big{});
+    // an expert cannot hold more pair rows than the call has tokens (a token selects it at most once)
+    const cudaError_t e = small_geometry(h, w) ? go(Gemm1Small{}) : go(Gemm1Big{});
     return e == cudaSuccess ? 1 : -1;
 }
 
-int launch_experts_gemm2_pair(const zeda_moe *h, int T, cudaStream_t s) {
+int launch_experts_gemm2_pair(const zeda_moe *h, const ExpertWork &w, cudaStream_t s) {
     const zeda_moe_config_t &c = h->cfg;
     const Workspace &ws = h->ws;
     const PairMaps *pm = static_cast<const PairMaps *>(h->pmaps);
     const int m_blocks = (c.d_model + 255) / 256;
     auto go = [&](auto k) {
-        return decltype(k)::launch(h, s, pm->w_down, pm->hmid, (const __nv_bfloat16 *)nullptr, 0, ws.counts, ws.offsets,
-                                   ws.ptile_expert, ws.ptile_row0, ws.pair_token, ws.meta, c.d_expert, c.d_model, m_blocks,
+        return decltype(k)::launch(h, s, pm->w_down, pm->hmid, (const __nv_bfloat16 *)nullptr, 0, w.counts, w.offsets,
+                                   w.tile_expert, w.tile_row0, w.pair_row, ws.meta, c.d_expert, c.d_model, m_blocks,
                                    ws.obuf, c.d_model);
     };
-    const cudaError_t e = T <= kSmallTokensMax ? go(Gemm2Small{}) : go(Gemm2Big{});
+    const cudaError_t e = small_geometry(h, w) ? go(Gemm2Small{}) : go(Gemm2Big{});
     return e == cudaSuccess ? 1 : -1;
 }
 

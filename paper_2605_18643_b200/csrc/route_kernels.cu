@@ -5,13 +5,11 @@
 
 #include <atomic>
 
-#include "zeda_internal.h"
+#include "expert_scan.cuh"
 
 namespace zeda {
 
 namespace {
-
-constexpr unsigned kFull = 0xffffffffu;
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -232,86 +230,6 @@ __device__ __forceinline__ void stage_ints(int32_t *__restrict__ dst, const int3
             const int i = i0 + u * blockDim.x;
             if (i < n) dst[i] = v[u];
         }
-    }
-}
-
-struct ScanShared {
-    int32_t cnt[kMaxCand];
-    int32_t off[kMaxCand + 1];
-    int32_t ptile[kMaxCand + 1];  // exclusive scan of the experts' tile counts
-};
-
-// From per-expert pair counts in sh.cnt: exclusive offsets, P, U, and the tile list of the expert
-// kernels (experts in id order, each with its tiles of kPairTileM rows in row order; the last tile of
-// an expert may be ragged).  Called by every thread of the CTA (blockDim.x >= 32); contains CTA
-// barriers.
-__device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, int total_slots,
-                                                   int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
-                                                   int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
-                                                   const WorkLists &wl, bool write_global = true,
-                                                   int list_part = 0, int list_parts = 1) {
-    if (threadIdx.x < 32) {
-        // warp 0 scans the per-expert sequences in steps of 32 with shuffle prefix sums
-        int base_off = 0, base_ptile = 0, active = 0, max_rows = 0;
-        for (int e0 = 0; e0 < n_real; e0 += 32) {
-            const int i = e0 + threadIdx.x;
-            const int c = (i < n_real) ? sh.cnt[i] : 0;
-            const int pt = (c + kPairTileM - 1) / kPairTileM;
-            int so = c, sp = pt;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int a = __shfl_up_sync(kFull, so, o);
-                const int q = __shfl_up_sync(kFull, sp, o);
-                if ((int)threadIdx.x >= o) { so += a; sp += q; }
-            }
-            if (i < n_real) {
-                sh.off[i] = base_off + so - c;
-                sh.ptile[i] = base_ptile + sp - pt;
-            }
-            base_off += __shfl_sync(kFull, so, 31);
-            base_ptile += __shfl_sync(kFull, sp, 31);
-            active += __popc(__ballot_sync(kFull, c > 0));
-            int mx = c;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(kFull, mx, o));
-            max_rows = max(max_rows, mx);
-        }
-        if (threadIdx.x == 0) {
-            sh.off[n_real] = base_off;
-            sh.ptile[n_real] = base_ptile;
-        }
-        if (threadIdx.x == 0 && write_global) {
-            meta[kMetaPairs] = base_off;
-            meta[kMetaActive] = active;
-            meta[kMetaZeroSlots] = total_slots - base_off;
-            meta[kMetaPairTiles] = base_ptile;
-            meta[kMetaMaxRows] = max_rows;
-            meta[kMetaNextItem1] = 0;
-            meta[kMetaNextItem2] = 0;
-            if (n_pairs_out) *n_pairs_out = base_off;
-        }
-    }
-    __syncthreads();
-    if (write_global) {  // (uniform over the CTA)
-        for (int e = threadIdx.x; e < n_real; e += blockDim.x) {
-            if (counts) counts[e] = sh.cnt[e];
-            offsets[e] = sh.off[e];
-        }
-        if (threadIdx.x == 0) offsets[n_real] = sh.off[n_real];
-    }
-    // Tile list: every CTA that runs this scan holds the same prefix sums, so the CTAs share the
-    // filling (part list_part of list_parts); a CTA outside that sharing passes list_parts = 0.
-    if (list_parts <= 0) return;
-    // entry i belongs to the expert whose first-entry index is the last one <= i
-    const int total = sh.ptile[n_real];
-    for (int i = list_part * blockDim.x + threadIdx.x; i < total; i += list_parts * blockDim.x) {
-        int lo = 0, hi = n_real;  // invariant: ptile[lo] <= i < ptile[hi]
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (sh.ptile[mid] <= i) lo = mid; else hi = mid;
-        }
-        wl.ptile_expert[i] = lo;
-        wl.ptile_row0[i] = (i - sh.ptile[lo]) * kPairTileM;
     }
 }
 
@@ -659,7 +577,23 @@ stats_final_kernel(const float *__restrict__ part, int nblk, int T, int K, int n
     }
 }
 
+// Per-token zero-expert ratio (Section 2.2, looked at per token in Section 4.1): the share of the
+// token's K slots that selected a zero expert.
+__global__ void __launch_bounds__(256)
+token_zero_share_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real, float *__restrict__ out) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    int zero = 0;
+    for (int k = 0; k < K; ++k) zero += topk_idx[(size_t)t * K + k] >= n_real ? 1 : 0;
+    out[t] = (float)zero / (float)K;
+}
+
 }  // namespace
+
+int launch_token_zero_share(const zeda_moe *h, int T, float *out, cudaStream_t s) {
+    token_zero_share_kernel<<<(T + 255) / 256, 256, 0, s>>>(h->ws.topk_idx, T, h->cfg.top_k, h->cfg.n_real, out);
+    return cudaGetLastError() == cudaSuccess ? 1 : -1;
+}
 
 int init_route_kernels(const zeda_moe *h) {
     const size_t smem = (size_t)kTok * h->cfg.d_model * sizeof(__nv_bfloat16);

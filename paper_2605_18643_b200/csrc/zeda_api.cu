@@ -37,6 +37,10 @@ bool config_ok(const zeda_moe_config_t *c, const char **why) {
     else if (c->gate_mode < 0 || c->gate_mode > 2) w = "unknown gate_mode";
     else if (c->expert_kind < 0 || c->expert_kind > 1) w = "unknown expert_kind";
     else if (c->flags & ~ZEDA_FLAG_NO_DEPENDENT_LAUNCH) w = "unknown flag";
+    else if (c->ep_size < 0 || c->ep_size > kMaxEpRanks) w = "ep_size must be in [0, 64]";
+    else if (c->ep_size >= 1 && (c->n_real % c->ep_size) != 0) w = "n_real must be a multiple of ep_size";
+    else if (c->ep_size >= 1 && (c->ep_rank < 0 || c->ep_rank >= c->ep_size)) w = "ep_rank outside [0, ep_size)";
+    else if (c->ep_size >= 1 && (c->max_recv_pairs < 1 || c->max_recv_pairs >= (1 << 27))) w = "max_recv_pairs must be in [1, 2^27)";
     if (why) *why = w;
     return w == nullptr;
 }
@@ -53,6 +57,11 @@ size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int
     const size_t n_cand = (size_t)c.n_real + c.n_zero;
     const size_t nblk = (c.max_tokens + kSortTokens - 1) / kSortTokens;
     const size_t tiles = slots / kPairTileM + c.n_real + 1;
+    // an expert-parallel handle holds n_local experts and sizes its pair buffers for the rows it may receive
+    const bool ep = c.ep_size >= 1;
+    const size_t n_local = ep ? (size_t)c.n_real / c.ep_size : (size_t)c.n_real;
+    const size_t pair_rows = ep ? (size_t)c.max_recv_pairs : slots;
+    const size_t ep_tiles = pair_rows / kPairTileM + n_local + 1;
     const size_t nblk_stats = (c.max_tokens + 63) / 64;
     Workspace w;
     w.topk_idx = (int32_t *)take(slots * 4);
@@ -69,15 +78,28 @@ size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int
     w.logits = (float *)take((size_t)router_part_rows(c.max_tokens) * n_cand * 4);
     w.stat_part = (float *)take(nblk_stats * 2 * n_cand * 4);
     // pair buffers carry one tile of slack rows so that a full tile may be read past the last pair
-    w.hmid = (__nv_bfloat16 *)take((slots + kPairTileM) * c.d_expert * 2);
-    w.obuf = (__nv_bfloat16 *)take((slots + kPairTileM) * c.d_model * 2);
+    w.hmid = (__nv_bfloat16 *)take((pair_rows + kPairTileM) * c.d_expert * 2);
+    w.obuf = (__nv_bfloat16 *)take((pair_rows + kPairTileM) * c.d_model * 2);
     w.router_split = (__nv_bfloat16 *)take((size_t)3 * router_split_pad((int)n_cand) * c.d_model * 2);
     w.x_stage = (__nv_bfloat16 *)take((size_t)c.max_tokens * c.d_model * 2);
     w.y_stage = (__nv_bfloat16 *)take((size_t)c.max_tokens * c.d_model * 2);
+    w.ep_counts = w.ep_offsets = w.ep_pair_row = w.ep_row_pos = w.ep_tile_expert = w.ep_tile_row0 = nullptr;
+    if (ep) {
+        w.ep_counts = (int32_t *)take(n_local * 4);
+        w.ep_offsets = (int32_t *)take((n_local + 1) * 4);
+        w.ep_pair_row = (int32_t *)take(pair_rows * 4);
+        w.ep_row_pos = (int32_t *)take(pair_rows * 4);
+        w.ep_tile_expert = (int32_t *)take(ep_tiles * 4);
+        w.ep_tile_row0 = (int32_t *)take(ep_tiles * 4);
+    }
     if (ws) *ws = w;
     if (max_tiles) *max_tiles = (int)tiles;
     return off;
 }
+
+// text for the sticky device-side error word
+const char kDeviceFailure[] = "a bounded device wait expired or a device-side check failed (code %d; 21 = the row count "
+                              "passed to zeda_ep_experts is not the sum of its count matrix)";
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -105,6 +127,7 @@ zeda_status_t check_call(zeda_moe_t *h, const void *in, int32_t T, const char *i
 int route_into(zeda_moe_t *h, const __nv_bfloat16 *x, const float *logits_in, int T, const RouteOut &out, cudaStream_t s,
                bool full_logits = false) {
     int n = 0, n_parts = 1;
+    h->last_routed_tokens = T;
     const float *logits = logits_in;
     if (!logits) {
         int r = launch_router_logits(h, x, T, h->ws.logits, s, full_logits ? nullptr : &n_parts);
@@ -121,6 +144,7 @@ zeda_status_t forward_device(zeda_moe_t *h, const __nv_bfloat16 *x, int T, __nv_
     const bool prof = h->profiling;
     auto mark = [&](int i) { if (prof) cudaEventRecord(h->ev[i], s); };
     mark(0);
+    h->last_routed_tokens = T;
     int n_parts = 1;
     int n = launch_router_logits(h, x, T, h->ws.logits, s, &n_parts);
     if (n < 0) return cuda_fail("router launch", cudaGetLastError());
@@ -130,11 +154,13 @@ zeda_status_t forward_device(zeda_moe_t *h, const __nv_bfloat16 *x, int T, __nv_
     if (r < 0) return cuda_fail("routing launch", cudaGetLastError());
     n += r;
     mark(2);
-    r = launch_experts_gemm1_pair(h, x, T, s);
+    const Workspace &ws = h->ws;
+    const ExpertWork work = {ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token, T * h->cfg.top_k};
+    r = launch_experts_gemm1_pair(h, x, work, s);
     if (r < 0) return cuda_fail("expert GEMM1 launch", cudaGetLastError());
     n += r;
     mark(3);
-    r = launch_experts_gemm2_pair(h, T, s);
+    r = launch_experts_gemm2_pair(h, work, s);
     if (r < 0) return cuda_fail("expert GEMM2 launch", cudaGetLastError());
     n += r;
     mark(4);
@@ -204,6 +230,9 @@ zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_
     h->sm_count = prop.multiProcessorCount;
     h->pdl = !(cfg->flags & ZEDA_FLAG_NO_DEPENDENT_LAUNCH);
     h->last_launches = 0;
+    h->last_routed_tokens = 0;
+    h->n_local = cfg->ep_size >= 1 ? cfg->n_real / cfg->ep_size : cfg->n_real;
+    h->pair_rows = cfg->ep_size >= 1 ? cfg->max_recv_pairs : cfg->max_tokens * cfg->top_k;
     h->pmaps = nullptr;
     h->router_maps = nullptr;
     h->profiling = false;
@@ -262,6 +291,7 @@ zeda_status_t zeda_router_logits(zeda_moe_t *h, const void *x, int32_t T, float 
 zeda_status_t zeda_moe_forward(zeda_moe_t *h, const void *x, int32_t T, void *y, void *stream) {
     zeda_status_t st = check_call(h, x, T, "x");
     if (st != ZEDA_OK || T == 0) return st;
+    if (h->cfg.ep_size >= 1) { set_error("an expert-parallel handle (ep_size >= 1) runs the layer through the zeda_ep_* calls"); return ZEDA_ERR_INVALID_ARG; }
     if (!y || !aligned16(y)) { set_error("y is NULL or not 16-byte aligned"); return ZEDA_ERR_INVALID_ARG; }
     const size_t bytes = (size_t)T * h->cfg.d_model * 2;
     const char *xb = static_cast<const char *>(x), *yb = static_cast<const char *>(y);
@@ -274,6 +304,7 @@ zeda_status_t zeda_moe_forward_host(zeda_moe_t *h, const void *x_host, int32_t T
     if (!h) { set_error("handle is NULL"); return ZEDA_ERR_INVALID_ARG; }
     if (T < 0 || T > h->cfg.max_tokens) { set_error("T=%d outside [0, max_tokens=%d]", T, h->cfg.max_tokens); return ZEDA_ERR_INVALID_ARG; }
     if (T == 0) return ZEDA_OK;
+    if (h->cfg.ep_size >= 1) { set_error("an expert-parallel handle (ep_size >= 1) runs the layer through the zeda_ep_* calls"); return ZEDA_ERR_INVALID_ARG; }
     if (!x_host || !y_host) { set_error("host buffer is NULL"); return ZEDA_ERR_INVALID_ARG; }
     cudaError_t e = cudaSetDevice(h->cfg.device);
     if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
@@ -290,6 +321,74 @@ zeda_status_t zeda_moe_forward_host(zeda_moe_t *h, const void *x_host, int32_t T
     return ZEDA_OK;
 }
 
+zeda_status_t zeda_ep_dispatch(zeda_moe_t *h, const void *x, int32_t T, void *send_rows, int32_t *send_counts,
+                               int32_t *expert_counts, void *stream) {
+    zeda_status_t st = check_call(h, x, T, "x");
+    if (st != ZEDA_OK) return st;
+    if (h->cfg.ep_size < 1) { set_error("the handle was not created for expert parallelism (ep_size = 0)"); return ZEDA_ERR_INVALID_ARG; }
+    if (!send_counts) { set_error("send_counts is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (T == 0) {  // nothing to route: this rank sends no rows
+        cudaError_t e = cudaMemsetAsync(send_counts, 0, sizeof(int32_t) * h->cfg.ep_size, s);
+        if (e == cudaSuccess && expert_counts) e = cudaMemsetAsync(expert_counts, 0, sizeof(int32_t) * h->cfg.n_real, s);
+        if (e == cudaSuccess) e = cudaMemsetAsync(h->ws.meta + kMetaPairs, 0, sizeof(int32_t), s);
+        return e == cudaSuccess ? ZEDA_OK : cuda_fail("cudaMemsetAsync", e);
+    }
+    if (!send_rows || !aligned16(send_rows)) { set_error("send_rows is NULL or not 16-byte aligned"); return ZEDA_ERR_INVALID_ARG; }
+    RouteOut none = {};
+    int n = route_into(h, static_cast<const __nv_bfloat16 *>(x), nullptr, T, none, s);
+    if (n < 0) return cuda_fail("routing launch", cudaGetLastError());
+    int r = launch_ep_pack(h, static_cast<const __nv_bfloat16 *>(x), T, static_cast<__nv_bfloat16 *>(send_rows), send_counts,
+                           expert_counts, s);
+    if (r < 0) return cuda_fail("pack launch", cudaGetLastError());
+    h->last_launches = n + r;
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_ep_experts(zeda_moe_t *h, const void *recv_rows, const int32_t *recv_counts, int32_t n_rows,
+                              void *out_rows, void *stream) {
+    if (!h) { set_error("handle is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    if (h->cfg.ep_size < 1) { set_error("the handle was not created for expert parallelism (ep_size = 0)"); return ZEDA_ERR_INVALID_ARG; }
+    if (n_rows < 0 || n_rows > h->cfg.max_recv_pairs) {
+        set_error("n_rows=%d outside [0, max_recv_pairs=%d]", n_rows, h->cfg.max_recv_pairs);
+        return ZEDA_ERR_INVALID_ARG;
+    }
+    if (n_rows == 0) return ZEDA_OK;
+    if (!recv_rows || !recv_counts || !out_rows || !aligned16(recv_rows) || !aligned16(out_rows)) {
+        set_error("recv_rows, recv_counts and out_rows are required; rows 16-byte aligned");
+        return ZEDA_ERR_INVALID_ARG;
+    }
+    cudaError_t e = cudaSetDevice(h->cfg.device);
+    if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int n = launch_ep_plan(h, recv_counts, n_rows, s);
+    if (n < 0) return cuda_fail("plan launch", cudaGetLastError());
+    const Workspace &ws = h->ws;
+    const ExpertWork work = {ws.ep_counts, ws.ep_offsets, ws.ep_tile_expert, ws.ep_tile_row0, ws.ep_pair_row, n_rows};
+    int r = launch_experts_gemm1_pair(h, static_cast<const __nv_bfloat16 *>(recv_rows), work, s);
+    if (r < 0) return cuda_fail("expert GEMM1 launch", cudaGetLastError());
+    n += r;
+    r = launch_experts_gemm2_pair(h, work, s);
+    if (r < 0) return cuda_fail("expert GEMM2 launch", cudaGetLastError());
+    n += r;
+    r = launch_ep_unsort(h, n_rows, static_cast<__nv_bfloat16 *>(out_rows), s);
+    if (r < 0) return cuda_fail("unsort launch", cudaGetLastError());
+    h->last_launches = n + r;
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_ep_combine(zeda_moe_t *h, const void *x, const void *back_rows, int32_t T, void *y, void *stream) {
+    zeda_status_t st = check_call(h, x, T, "x");
+    if (st != ZEDA_OK || T == 0) return st;
+    if (h->cfg.ep_size < 1) { set_error("the handle was not created for expert parallelism (ep_size = 0)"); return ZEDA_ERR_INVALID_ARG; }
+    if (!y || !aligned16(y) || !back_rows || !aligned16(back_rows)) { set_error("back_rows and y are required, 16-byte aligned"); return ZEDA_ERR_INVALID_ARG; }
+    int r = launch_combine_rows(h, static_cast<const __nv_bfloat16 *>(back_rows), static_cast<const __nv_bfloat16 *>(x), T,
+                                static_cast<__nv_bfloat16 *>(y), static_cast<cudaStream_t>(stream));
+    if (r < 0) return cuda_fail("combine launch", cudaGetLastError());
+    h->last_launches = r;
+    return ZEDA_OK;
+}
+
 zeda_status_t zeda_moe_stats(zeda_moe_t *h, const void *x, int32_t T, float *f, float *p_mean, float *out, void *stream) {
     zeda_status_t st = check_call(h, x, T, "x");
     if (st != ZEDA_OK || T == 0) return st;
@@ -300,6 +399,21 @@ zeda_status_t zeda_moe_stats(zeda_moe_t *h, const void *x, int32_t T, float *f, 
     int r = launch_stats(h, h->ws.logits, h->ws.topk_idx, T, f, p_mean, out, s);
     if (r < 0) return cuda_fail("stats launch", cudaGetLastError());
     h->last_launches = n + r;
+    return ZEDA_OK;
+}
+
+zeda_status_t zeda_moe_token_zero_share(zeda_moe_t *h, int32_t T, float *r_ze, void *stream) {
+    if (!h) { set_error("handle is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    if (T == 0) return ZEDA_OK;
+    if (T < 0 || T != h->last_routed_tokens) {
+        set_error("T=%d is not the token count of the last routing pass on this handle (%d)", T, h->last_routed_tokens);
+        return ZEDA_ERR_INVALID_ARG;
+    }
+    if (!r_ze) { set_error("r_ze is NULL"); return ZEDA_ERR_INVALID_ARG; }
+    cudaError_t e = cudaSetDevice(h->cfg.device);
+    if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
+    if (launch_token_zero_share(h, T, r_ze, static_cast<cudaStream_t>(stream)) < 0)
+        return cuda_fail("token_zero_share launch", cudaGetLastError());
     return ZEDA_OK;
 }
 
@@ -317,7 +431,7 @@ zeda_status_t zeda_moe_last_counters(zeda_moe_t *h, int64_t out[4], void *stream
     out[1] = meta[kMetaActive];
     out[2] = meta[kMetaZeroSlots];
     out[3] = h->last_launches;
-    if (meta[kMetaError] != 0) { set_error("a bounded device wait expired (code %d)", meta[kMetaError]); return ZEDA_ERR_TIMEOUT; }
+    if (meta[kMetaError] != 0) { set_error(kDeviceFailure, meta[kMetaError]); return ZEDA_ERR_TIMEOUT; }
     return ZEDA_OK;
 }
 
@@ -379,7 +493,7 @@ zeda_status_t zeda_moe_destroy(zeda_moe_t *h) {
         cudaError_t e = cudaDeviceSynchronize();
         if (e == cudaSuccess) e = cudaMemcpy(&err, h->ws.meta + kMetaError, 4, cudaMemcpyDeviceToHost);
         if (e != cudaSuccess) st = cuda_fail("zeda_moe_destroy", e);
-        else if (err != 0) { set_error("a bounded device wait expired (code %d)", err); st = ZEDA_ERR_TIMEOUT; }
+        else if (err != 0) { set_error(kDeviceFailure, err); st = ZEDA_ERR_TIMEOUT; }
     }
     for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
     if (h->pmaps) free(h->pmaps);

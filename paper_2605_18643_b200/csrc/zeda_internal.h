@@ -13,6 +13,7 @@ constexpr int kMaxCand = 512;       // N + N_Z limit (16 logits per lane in the 
 constexpr int kMaxTopK = 16;
 constexpr int kSortTokens = 128;    // tokens per CTA in the counting sort (histogram / placement)
 constexpr int kPairTileM = 256;     // pair rows per tile of the expert kernels (one CTA pair, N <= 256)
+constexpr int kMaxEpRanks = 64;     // expert-parallel group size limit
 
 // Device-resident counters of one call.
 enum MetaSlot {
@@ -46,6 +47,20 @@ struct Workspace {
     __nv_bfloat16 *router_split; // [3][pad128(N+N_Z)][d] bf16 hi/mid/lo pieces of the router rows
     __nv_bfloat16 *x_stage;// [maxT, d]
     __nv_bfloat16 *y_stage;// [maxT, d]
+    // expert-parallel handles only: the plan of the rows received from the group
+    int32_t *ep_counts;      // [N_local] received pairs per local expert
+    int32_t *ep_offsets;     // [N_local + 1]
+    int32_t *ep_pair_row;    // [maxR] sorted position -> received row
+    int32_t *ep_row_pos;     // [maxR] received row -> sorted position
+    int32_t *ep_tile_expert; // [maxR / kPairTileM + N_local + 1]
+    int32_t *ep_tile_row0;
+};
+
+// What one launch of the expert kernels works on: per-expert counts and offsets of the pair rows,
+// the tile list, and for GEMM1 the row of the activation matrix that each pair row reads.
+struct ExpertWork {
+    const int32_t *counts, *offsets, *tile_expert, *tile_row0, *pair_row;
+    int rows_bound;  // upper bound of the pair rows of a call (host-side; picks the kernel geometry)
 };
 
 // Device-side tile list written by the expert scan: experts in id order, each with its tiles of at
@@ -75,11 +90,14 @@ struct zeda_moe {
     zeda::Workspace ws;
     int sm_count;
     int max_tiles;
+    int n_local;    // experts whose weights this handle holds (n_real unless expert-parallel)
+    int pair_rows;  // capacity of the pair buffers (max_tokens * top_k, or max_recv_pairs)
     int last_launches;
     void *pmaps;  // host-side tensor maps of the expert kernels (owned)
     void *router_maps;  // host-side tensor map of the split router weights (owned)
     bool profiling;
     bool profiled_last;
+    int last_routed_tokens;  // T of the most recent routing pass on this handle
     cudaEvent_t ev[ZEDA_STAGE_COUNT + 1];
 };
 
@@ -108,8 +126,16 @@ inline long long router_part_rows(long long max_tokens) {
 int router_split_factor(const zeda_moe *h, int T);
 int launch_router_logits_tile(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, int split, cudaStream_t s);
 int init_pair_kernels(zeda_moe *h);
-int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, int T, cudaStream_t s);
-int launch_experts_gemm2_pair(const zeda_moe *h, int T, cudaStream_t s);
+int launch_token_zero_share(const zeda_moe *h, int T, float *out, cudaStream_t s);
+int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, const ExpertWork &w, cudaStream_t s);
+int launch_experts_gemm2_pair(const zeda_moe *h, const ExpertWork &w, cudaStream_t s);
+// expert-parallel pieces (expert_parallel.cu)
+int launch_ep_pack(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *send_rows, int32_t *send_counts,
+                   int32_t *expert_counts, cudaStream_t s);
+int launch_ep_plan(const zeda_moe *h, const int32_t *recv_counts, int n_rows, cudaStream_t s);
+int launch_ep_unsort(const zeda_moe *h, int n_rows, __nv_bfloat16 *out_rows, cudaStream_t s);
+int launch_combine_rows(const zeda_moe *h, const __nv_bfloat16 *rows, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y,
+                        cudaStream_t s);
 int launch_wait_selftest(const zeda_moe *h, long long limit_cycles, cudaStream_t s);
 int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s);
 

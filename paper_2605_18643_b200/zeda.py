@@ -24,8 +24,9 @@ FLAG_NONE, FLAG_NO_DEPENDENT_LAUNCH = 0, 4
 EXPORTS = (
     "zeda_moe_workspace_bytes", "zeda_moe_create", "zeda_route", "zeda_route_from_logits",
     "zeda_router_logits", "zeda_moe_forward", "zeda_moe_forward_host", "zeda_moe_stats",
-    "zeda_moe_last_counters", "zeda_moe_set_profiling", "zeda_moe_stage_ms", "zeda_residual_rmsnorm",
+    "zeda_moe_token_zero_share", "zeda_moe_last_counters", "zeda_moe_set_profiling", "zeda_moe_stage_ms", "zeda_residual_rmsnorm",
     "zeda_moe_selftest_wait", "zeda_moe_clear_error",
+    "zeda_ep_dispatch", "zeda_ep_experts", "zeda_ep_combine",
     "zeda_compact_static", "zeda_moe_destroy", "zeda_last_error", "zeda_version",
 )
 
@@ -33,7 +34,7 @@ EXPORTS = (
 class Config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "d_model", "d_expert", "n_real", "n_zero", "top_k", "max_tokens", "gate_mode", "expert_kind",
-        "device", "flags")]
+        "device", "flags", "ep_size", "ep_rank", "max_recv_pairs")]
 
 
 class ZedaError(RuntimeError):
@@ -65,6 +66,8 @@ def _load() -> ctypes.CDLL:
     lib.zeda_moe_forward_host.argtypes = [vp, vp, i32, vp, vp]
     lib.zeda_moe_stats.restype = i32
     lib.zeda_moe_stats.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    lib.zeda_moe_token_zero_share.restype = i32
+    lib.zeda_moe_token_zero_share.argtypes = [vp, i32, vp, vp]
     lib.zeda_moe_last_counters.restype = i32
     lib.zeda_moe_last_counters.argtypes = [vp, ctypes.POINTER(ctypes.c_int64), vp]
     lib.zeda_moe_set_profiling.restype = i32
@@ -77,6 +80,12 @@ def _load() -> ctypes.CDLL:
     lib.zeda_moe_clear_error.argtypes = [vp, vp]
     lib.zeda_residual_rmsnorm.restype = i32
     lib.zeda_residual_rmsnorm.argtypes = [vp, vp, vp, i32, i32, ctypes.c_float, vp]
+    lib.zeda_ep_dispatch.restype = i32
+    lib.zeda_ep_dispatch.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    lib.zeda_ep_experts.restype = i32
+    lib.zeda_ep_experts.argtypes = [vp, vp, vp, i32, vp, vp]
+    lib.zeda_ep_combine.restype = i32
+    lib.zeda_ep_combine.argtypes = [vp, vp, vp, i32, vp, vp]
     lib.zeda_compact_static.restype = i32
     lib.zeda_compact_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.zeda_moe_destroy.restype = i32
@@ -155,18 +164,23 @@ class ZedaMoE:
     def __init__(self, router_w: torch.Tensor, router_bias: Optional[torch.Tensor], w_gate_up: torch.Tensor,
                  w_down: torch.Tensor, n_real: int, n_zero: int, top_k: int, max_tokens: int,
                  gate_mode: int = GATE_TOPK_NORM, expert_kind: int = EXPERT_ZERO, flags: int = FLAG_NONE,
-                 workspace: Optional[torch.Tensor] = None):
+                 workspace: Optional[torch.Tensor] = None, ep_size: int = 0, ep_rank: int = 0,
+                 max_recv_pairs: int = 0):
+        """ep_size >= 1 makes an expert-parallel handle: the weight tensors then hold only the
+        experts [ep_rank * N/G, (ep_rank + 1) * N/G) of the layer."""
         dev = router_w.device
         assert dev.type == "cuda", "weights must live on a CUDA device"
         d = router_w.shape[1]
         He = w_down.shape[2]
+        n_local = n_real // ep_size if ep_size >= 1 else n_real
         assert router_w.dtype == torch.float32 and router_w.is_contiguous() and router_w.shape == (n_real + n_zero, d)
-        assert w_gate_up.dtype == torch.bfloat16 and w_gate_up.is_contiguous() and w_gate_up.shape == (n_real, 2 * He, d)
-        assert w_down.dtype == torch.bfloat16 and w_down.is_contiguous() and w_down.shape == (n_real, d, He)
+        assert w_gate_up.dtype == torch.bfloat16 and w_gate_up.is_contiguous() and w_gate_up.shape == (n_local, 2 * He, d)
+        assert w_down.dtype == torch.bfloat16 and w_down.is_contiguous() and w_down.shape == (n_local, d, He)
         if router_bias is not None:
             assert router_bias.dtype == torch.float32 and router_bias.is_contiguous() and router_bias.shape == (n_real + n_zero,)
         self.cfg = Config(d, He, n_real, n_zero, top_k, max_tokens, gate_mode, expert_kind,
-                          dev.index if dev.index is not None else torch.cuda.current_device(), flags)
+                          dev.index if dev.index is not None else torch.cuda.current_device(), flags,
+                          ep_size, ep_rank, max_recv_pairs)
         need = workspace_bytes(self.cfg)
         if need == 0:
             raise ZedaError(ERR_INVALID_ARG, last_error())
@@ -233,6 +247,42 @@ class ZedaMoE:
         _check(lib.zeda_moe_forward_host(self._h, _ptr(x_host), T, _ptr(out_host), _stream(self.device)))
         return out_host
 
+    # -- expert parallelism -------------------------------------------------------------------
+    def ep_dispatch(self, x: torch.Tensor, send_rows: Optional[torch.Tensor] = None):
+        """zeda_ep_dispatch: routes x and packs the rows of the surviving pairs.  Returns device
+        tensors (send_rows [T*K, d], send_counts [G], expert_counts [N])."""
+        T = self._check_x(x)
+        G = max(1, self.cfg.ep_size)
+        if send_rows is None:
+            send_rows = torch.empty((T * self.K, self.d), dtype=torch.bfloat16, device=self.device)
+        send_counts = torch.empty(G, dtype=torch.int32, device=self.device)
+        expert_counts = torch.empty(self.E, dtype=torch.int32, device=self.device)
+        _check(lib.zeda_ep_dispatch(self._h, _ptr(x), T, _ptr(send_rows), _ptr(send_counts), _ptr(expert_counts),
+                                    _stream(self.device)))
+        return send_rows, send_counts, expert_counts
+
+    def ep_experts(self, recv_rows: torch.Tensor, recv_counts: torch.Tensor, n_rows: int,
+                   out_rows: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """zeda_ep_experts: this rank's experts on the first n_rows rows of recv_rows; recv_counts is
+        the device matrix [G, N/G] of rows per (source rank, local expert)."""
+        assert recv_rows.dtype == torch.bfloat16 and recv_rows.is_contiguous() and recv_rows.shape[1] == self.d
+        assert recv_counts.dtype == torch.int32 and recv_counts.is_contiguous()
+        assert recv_rows.shape[0] >= n_rows
+        if out_rows is None:
+            out_rows = torch.empty((max(n_rows, 1), self.d), dtype=torch.bfloat16, device=self.device)
+        _check(lib.zeda_ep_experts(self._h, _ptr(recv_rows), _ptr(recv_counts), int(n_rows), _ptr(out_rows),
+                                   _stream(self.device)))
+        return out_rows
+
+    def ep_combine(self, x: torch.Tensor, back_rows: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """zeda_ep_combine: Eq. 1 on the expert outputs that came back, in the order of send_rows."""
+        T = self._check_x(x)
+        assert back_rows.dtype == torch.bfloat16 and back_rows.is_contiguous() and back_rows.shape[1] == self.d
+        if out is None:
+            out = torch.empty_like(x)
+        _check(lib.zeda_ep_combine(self._h, _ptr(x), _ptr(back_rows), T, _ptr(out), _stream(self.device)))
+        return out
+
     def stats(self, x: torch.Tensor):
         """zeda_moe_stats: (f [N+N_Z], p_mean [N+N_Z], out [4] = r_ZE, sum f_i P_i, f_E P_E, f_Z P_Z)."""
         T = self._check_x(x)
@@ -242,6 +292,13 @@ class ZedaMoE:
         o = torch.empty(4, dtype=torch.float32, device=self.device)
         _check(lib.zeda_moe_stats(self._h, _ptr(x), T, _ptr(f), _ptr(p), _ptr(o), _stream(self.device)))
         return f, p, o
+
+    def token_zero_share(self, T: int) -> torch.Tensor:
+        """zeda_moe_token_zero_share: per-token share of the K slots on zero experts, for the T tokens of
+        the last routing call on this handle."""
+        out = torch.empty(T, dtype=torch.float32, device=self.device)
+        _check(lib.zeda_moe_token_zero_share(self._h, T, _ptr(out), _stream(self.device)))
+        return out
 
     def last_counters(self):
         """(P, U, zero slots, kernel launches) of the last call; synchronises the current stream."""

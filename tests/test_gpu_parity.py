@@ -242,6 +242,23 @@ def test_routing_statistics(zeda):
     m.close()
 
 
+def test_per_token_zero_share(zeda):
+    # the decode recipe spreads the per-token zero share over 0..100 %
+    wl = inputs.decode()
+    dev = torch.device("cuda:0")
+    m = zeda.from_workload(wl, dev)
+    x = wl.x.to(dev)
+    m.forward(x)
+    r = m.token_zero_share(wl.T).cpu().numpy()
+    _, idx, *_ = oracle_route(wl)
+    want = oracle.token_zero_share(idx, wl.E)
+    assert np.array_equal(r, want.astype(np.float32))
+    assert r.min() == 0.0 and r.max() == 1.0 and abs(r.mean() - wl.zero_fraction) < 1e-6
+    with pytest.raises(zeda.ZedaError):
+        m.token_zero_share(wl.T - 1)               # not the size of the last routing call
+    m.close()
+
+
 def test_tensor_core_router_path(zeda):
     # T >= 256 sends the router GEMM to the tensor cores (three-way bf16 split of the fp32 rows)
     for T in (256, 1000):

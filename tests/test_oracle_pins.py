@@ -402,3 +402,21 @@ def test_residual_add_is_the_correctly_rounded_sum():
         e = np.floor(np.log2(abs(float(exact))))
         ulp = fractions.Fraction(2) ** int(e - 7)
         assert abs(g - exact) <= ulp / 2, (float(a[0, i]), float(b[0, i]), float(g))
+
+
+def test_token_zero_share_counts_slots_and_averages_to_r_ze():
+    # Section 2.2 / 4.1: per token, the share of its K slots on zero experts; its batch mean is r_ZE
+    rng = np.random.default_rng(3)
+    E, Z, K, T = 6, 5, 4, 300
+    l = rng.standard_normal((T, E + Z)).astype(np.float32)
+    l[0, E:] += 100.0          # token 0: every slot on a zero expert
+    l[1, :E] += 100.0          # token 1: none
+    idx, _ = oracle.route(l, E, Z, K)
+    r = oracle.token_zero_share(idx, E)
+    assert r[0] == 1.0 and r[1] == 0.0
+    assert set(np.unique(r * K)).issubset(set(range(K + 1)))             # multiples of 1/K
+    brute = np.array([sum(1 for i in row if i >= E) / K for row in idx])
+    assert np.array_equal(r, brute)
+    s = oracle.stats(l, idx, E, Z)
+    assert abs(r.mean() - s["r_ze"]) < 1e-15
+    assert np.array_equal(oracle.token_zero_share(np.zeros((3, 2), dtype=np.int32), 1), np.zeros(3))   # Z = 0 layer
