@@ -397,6 +397,84 @@ def run_stack(args, peaks, peaks_kind, dev, world, rank, barrier, dist):
         m.close()
 
 
+def run_ep(args, peaks, peaks_kind, dev, world, rank, barrier, dist):
+    """--workload ep: the prefill layer with its experts partitioned over the N ranks (expert parallel)
+    and the tokens data-parallel, T tokens per rank.  One step = dispatch (route, drop zero slots, pack),
+    all-to-all of the surviving rows, local experts, all-to-all back, combine.  With N = 1 the exchange
+    is a loopback."""
+    from paper_2605_18643_b200 import ep, zeda
+    wl = inputs.prefill()
+    G = world
+    if wl.E % G:
+        raise SystemExit("--workload ep needs a rank count that divides %d experts" % wl.E)
+    n_local = wl.E // G
+    x_cpu = rank_tokens(wl, rank)
+    wgu = wl.w_gate_up[rank * n_local:(rank + 1) * n_local].contiguous().to(dev)
+    wd = wl.w_down[rank * n_local:(rank + 1) * n_local].contiguous().to(dev)
+    m = zeda.ZedaMoE(wl.router_w.to(dev), wl.router_bias.to(dev), wgu, wd, wl.E, wl.Z, wl.K, wl.T, ep_size=G,
+                     ep_rank=rank, max_recv_pairs=G * wl.T * wl.K)
+    layer = ep.ExpertParallelMoE(m, ep.TorchDistExchange() if dist is not None else ep.LoopbackExchange())
+    x = x_cpu.to(dev)
+    y = torch.empty_like(x)
+    flush = L2Flush(dev)
+    clocks = ClockSampler(dev.index or 0)
+    clocks.start()
+    for _ in range(args.warmup):
+        flush.zero_()
+        layer.forward(x, y)
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    barrier()
+    torch.cuda.synchronize()
+    for i in range(args.steps):
+        flush.zero_()
+        starts[i].record()
+        layer.forward(x, y)
+        ends[i].record()
+    torch.cuda.synchronize()
+    barrier()
+    total_ms = sum(a.elapsed_time(b) for a, b in zip(starts, ends))
+    per_phase = []
+    layer.forward(x, y, launches=per_phase)            # one more step, untimed: kernels per phase
+    launches = sum(per_phase)
+    R, U_local, _, _ = m.last_counters()               # pair rows this rank's experts processed, its active experts
+    x_pin = x_cpu.pin_memory()
+    y_pin = torch.empty_like(x_pin).pin_memory()
+    e2e_s = 0.0
+    for i in range(args.warmup + args.steps):
+        flush.zero_()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        x.copy_(x_pin, non_blocking=True)
+        layer.forward(x, y)
+        y_pin.copy_(y, non_blocking=True)
+        torch.cuda.synchronize()
+        if i >= args.warmup:
+            e2e_s += time.perf_counter() - t0
+    barrier()
+    clock_info = clocks.stop()
+    total_ms, e2e_s, rows_max = max_over_ranks([total_ms, e2e_s, float(R)], dist, dev)
+    if rank == 0:
+        ms = total_ms / args.steps
+        line = {
+            "metric": METRIC, "value": job_tokens_per_s(world, wl.T, ms), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "ep", "T_per_rank": wl.T, "d": wl.d, "d_expert": wl.He, "n_real": wl.E, "n_zero": wl.Z,
+                       "top_k": wl.K, "zero_slot_fraction": round(wl.zero_fraction, 4), "seed": 0,
+                       "pair_rows_rank0": int(R), "pair_rows_max_over_ranks": int(rows_max), "active_experts_rank0": int(U_local),
+                       "l2": L2_NOTE, "parallelism": "ep%d: experts over %d ranks, tokens data-parallel, zero slots dropped "
+                                                     "before the all-to-all" % (G, G)},
+            "clocks": clock_info,
+            "e2e": {"value": world * wl.T * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": wl.T * wl.d * 2,
+                    "d2h_bytes_per_step": wl.T * wl.d * 2, "ms_per_step": 1e3 * e2e_s / args.steps},
+            "gpu_launches": launches * args.steps,
+            "roofline": None,
+        }
+        print(json.dumps(line))
+    m.close()
+
+
 class DeviceWeights:
     """Device copies of expert weights, shared between the handles of one run (the zero-expert layer,
     its static reference, the decode batch on the same layer): 1.2 GB is copied once."""
@@ -528,7 +606,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="prefill",
                     help="prefill (default; carries the decode batch on the same layer as a nested object), decode, "
-                         "tiny, net, glm, sweepNN, prefill_fNN, stack")
+                         "tiny, net, glm, sweepNN, prefill_fNN, stack, ep (experts over the ranks)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-static", action="store_true")
     ap.add_argument("--no-decode", action="store_true", help="prefill only: skip the nested decode measurement")
@@ -559,8 +637,8 @@ def main():
     from paper_2605_18643_b200 import zeda  # raises if libzeda.so is missing
 
     peaks, peaks_kind = load_peaks()
-    if args.workload == "stack":
-        run_stack(args, peaks, peaks_kind, dev, world, rank, barrier, dist)
+    if args.workload in ("stack", "ep"):
+        (run_stack if args.workload == "stack" else run_ep)(args, peaks, peaks_kind, dev, world, rank, barrier, dist)
         if dist is not None:
             dist.destroy_process_group()
         return

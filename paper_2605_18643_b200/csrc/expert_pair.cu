@@ -331,7 +331,12 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                     const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
                     ok = __all_sync(0xffffffffu, mbar_wait(bar_gfull + 8 * s, ph, abort_flag));
                     if (!ok) break;
-                    if (elect_one()) mbar_arrive_cluster(full0 + 8 * s);
+                    if (elect_one()) {
+                        // the rows were written by cp.async (generic proxy) and are read by the MMA through
+                        // the async proxy: order the two before the stage is handed over
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        mbar_arrive_cluster(full0 + 8 * s);
+                    }
                     __syncwarp();
                 }
             }

@@ -72,6 +72,18 @@ class TorchDistExchange:
         return out
 
 
+class LoopbackExchange:
+    """The exchange of a group of one: counts and rows stay where they are."""
+
+    rank, size = 0, 1
+
+    def counts(self, expert_counts: torch.Tensor) -> torch.Tensor:
+        return expert_counts.view(1, -1).contiguous()
+
+    def rows(self, send: torch.Tensor, send_splits: Sequence[int], recv_splits: Sequence[int]) -> torch.Tensor:
+        return send
+
+
 class ExpertParallelMoE:
     """One rank of an expert-parallel zero-expert MoE layer on a GPU.
 
@@ -85,9 +97,13 @@ class ExpertParallelMoE:
         self.G = moe.cfg.ep_size
         assert self.G >= 1 and (exchange is None or exchange.size == self.G)
 
-    def forward(self, x: torch.Tensor, out: torch.Tensor = None) -> torch.Tensor:
+    def forward(self, x: torch.Tensor, out: torch.Tensor = None, launches: list = None) -> torch.Tensor:
+        """One layer call of this rank.  `launches`, if given, receives the number of library kernels
+        each of the three device phases enqueued (costs three host synchronisations)."""
         m = self.moe
         send_rows, send_counts, expert_counts = m.ep_dispatch(x)
+        if launches is not None:
+            launches.append(m.last_counters()[3])
         recv_counts = self.x.counts(expert_counts)
         # the one host synchronisation of the call: the all-to-all needs its split sizes on the host
         send_splits = [int(v) for v in send_counts.tolist()]
@@ -96,8 +112,13 @@ class ExpertParallelMoE:
             raise RuntimeError("rank receives %d pair rows, handle was sized for %d" % (n_rows, m.cfg.max_recv_pairs))
         recv_rows = self.x.rows(send_rows, send_splits, recv_splits)
         out_rows = m.ep_experts(recv_rows, recv_counts, n_rows)
+        if launches is not None:
+            launches.append(m.last_counters()[3])
         back_rows = self.x.rows(out_rows, recv_splits, send_splits)
-        return m.ep_combine(x, back_rows, out)
+        y = m.ep_combine(x, back_rows, out)
+        if launches is not None:
+            launches.append(m.last_counters()[3])
+        return y
 
 
 def forward_group_in_one_process(ranks: Sequence["ExpertParallelMoE"], xs: Sequence[torch.Tensor]):
