@@ -610,6 +610,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-static", action="store_true")
     ap.add_argument("--no-decode", action="store_true", help="prefill only: skip the nested decode measurement")
+    ap.add_argument("--no-sweep", action="store_true", help="prefill only: skip the nested zero-fraction sweep")
     ap.add_argument("--layers", type=int, default=48, help="layers of --workload stack")
     ap.add_argument("--stack-tokens", type=int, default=4096, help="tokens per pass of --workload stack")
     args = ap.parse_args()
@@ -661,6 +662,16 @@ def main():
                            e2e=False, static=not args.no_static)
         nested = (wd_, rd, clocks_d.stop())
 
+    sweep = None
+    if headline and not args.no_sweep and not args.no_static:
+        # layer time against the zero-routed share at the prefill size: 0 (the static layer) and the
+        # headline's own share are measured above; two more points with the same x and expert weights
+        sweep = {}
+        for f in (0.25, 0.75):
+            wf = inputs.prefill(zero_fraction=f)
+            rf = measure_layer(zeda, weights, wf, rank_tokens(wf, rank), args, flush, barrier, dist, dev, e2e=False, static=False)
+            sweep[f] = (wf, rf)
+
     if rank == 0:
         rep = layer_report(wl, args.workload, r, world, args.steps, peaks, peaks_kind)
         line = {
@@ -682,6 +693,17 @@ def main():
             dec["clocks"] = clk
             dec["gpu_launches"] = rd["launches"] * args.steps
             line["decode"] = dec
+        if sweep:
+            # time relative to the static layer next to the share of slots that still reach an expert
+            t0 = line["static_reference"]["ms_per_step"]
+            pts = [{"zero_slot_fraction": 0.0, "P": line["static_reference"]["P"], "ms_per_step": t0}]
+            for f, (wf, rf) in sorted(list(sweep.items()) + [(wl.zero_fraction, (wl, r))], key=lambda kv: kv[0]):
+                pts.append({"zero_slot_fraction": round(wf.zero_fraction, 4), "P": rf["P"], "U": rf["U"],
+                            "ms_per_step": rf["ms_per_step"]})
+            for p_ in pts:
+                p_["time_vs_static"] = p_["ms_per_step"] / t0
+                p_["real_slot_share"] = 1.0 - p_["zero_slot_fraction"]
+            line["zero_fraction_sweep"] = pts
         if not args.no_cpu_baseline:
             v, dt, cores, desc = oracle_tokens_per_s(wl, 64, min_seconds=10.0, max_passes=400)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
