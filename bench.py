@@ -84,6 +84,8 @@ def make_workload(name: str):
         return inputs.prefill()
     if name == "tiny":
         return inputs.tiny()
+    if name == "hot4":     # 32,768 pairs on four experts: full tiles only, weights resident in L2 (kernel ceiling)
+        return inputs.make_layer("hot4", T=8192, d=2048, He=768, E=4, Z=0, K=4, zero_fraction=None)
     if name == "net":      # the paper's iso-FLOP static baseline: no zero experts, K/2 slots
         return net_reference(inputs.prefill())
     if name == "glm":      # second adapted model's expert counts at the prefill size
@@ -606,7 +608,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="prefill",
                     help="prefill (default; carries the decode batch on the same layer as a nested object), decode, "
-                         "tiny, net, glm, sweepNN, prefill_fNN, stack, ep (experts over the ranks)")
+                         "tiny, net, glm, hot4, sweepNN, prefill_fNN, stack, ep (experts over the ranks)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-static", action="store_true")
     ap.add_argument("--no-decode", action="store_true", help="prefill only: skip the nested decode measurement")
