@@ -141,8 +141,7 @@ __device__ __forceinline__ void topk_gate_token(const float *__restrict__ row, i
         if (u == 0x80000000u) u = 0u;  // -0 and +0 are equal logits: the lower id decides between them
         key[r] = (r * 32 + lane < n_cand) ? ((u & 0x80000000u) ? ~u : (u | 0x80000000u)) : 0u;
     }
-    float my_p = 0.f;
-    float sum_sel = 0.f, sum_real = 0.f;
+    unsigned my_key = 0u;
     my_idx = -1;
     for (int k = 0; k < K; ++k) {
         unsigned lm = key[0];
@@ -157,12 +156,16 @@ __device__ __forceinline__ void topk_gate_token(const float *__restrict__ row, i
 #pragma unroll
         for (int r = 0; r < RPL; ++r)
             if (r * 32 + lane == bj) key[r] = 0u;
-        const float bv = __uint_as_float((gm & 0x80000000u) ? (gm & 0x7fffffffu) : ~gm);
-        const float p = expf(bv - m) / den;
-        sum_sel += p;
-        if (bj < n_real) sum_real += p;
-        if (lane == k) { my_idx = bj; my_p = p; }
+        if (lane == k) { my_idx = bj; my_key = gm; }
     }
+    // lane k < K holds slot k: its softmax probability, then the sums over the selected slots
+    float my_p = 0.f;
+    if (lane < K) {
+        const float bv = __uint_as_float((my_key & 0x80000000u) ? (my_key & 0x7fffffffu) : ~my_key);
+        my_p = expf(bv - m) / den;
+    }
+    const float sum_sel = warp_sum(my_p);
+    const float sum_real = warp_sum(my_idx >= 0 && my_idx < n_real ? my_p : 0.f);
     my_w = my_p;
     if (gate_mode == ZEDA_GATE_TOPK_NORM) my_w = my_p / sum_sel;
     else if (gate_mode == ZEDA_GATE_RENORM_REAL) my_w = (my_idx < n_real && sum_real > 0.f) ? my_p / sum_real : 0.f;
