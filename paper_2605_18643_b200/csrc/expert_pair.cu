@@ -63,14 +63,14 @@ struct Item {
     int e, pos0, n, mb;
 };
 
-__device__ __forceinline__ Item load_item(long long item, int m_blocks, const int32_t *tile_expert,
+__device__ __forceinline__ Item load_item(long long item, int m_blocks, int tile_rows, const int32_t *tile_expert,
                                           const int32_t *tile_row0, const int32_t *counts, const int32_t *offsets) {
     Item it;
     const int tile = (int)(item / m_blocks);
     it.mb = (int)(item % m_blocks);
     it.e = tile_expert[tile];
     const int r0 = tile_row0[tile];
-    it.n = min(kPairTileM, counts[it.e] - r0);
+    it.n = min(tile_rows, counts[it.e] - r0);
     it.pos0 = offsets[it.e] + r0;
     return it;
 }
@@ -147,7 +147,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                         const int32_t *__restrict__ offsets, const int32_t *__restrict__ tile_expert,
                         const int32_t *__restrict__ tile_row0, const int32_t *__restrict__ pair_token,
                         int32_t *__restrict__ meta, int kdim, int out_rows, int m_blocks,
-                        __nv_bfloat16 *__restrict__ out, int out_ld) {
+                        __nv_bfloat16 *__restrict__ out, int out_ld, int tile_rows) {
     static_assert(STAGES <= 10, "the item queue's depth assumes at most 10 ring stages");
     constexpr int kStageBytes = kATileBytes + HALF_MAX * kRowBytes;
     constexpr int kTmemCols = ACC_BUFS * kAccCols;
@@ -370,7 +370,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                     const long long item = atomicAdd(counter, 1);
                     Item it = {0, 0, 1, 0};
                     end = item >= n_items;
-                    if (!end) it = load_item(item, m_blocks, tile_expert, tile_row0, counts, offsets);
+                    if (!end) it = load_item(item, m_blocks, tile_rows, tile_expert, tile_row0, counts, offsets);
                     const unsigned long long rec = pack_item(seq, end, it);
                     asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(peer_queue + 8 * (seq % kItemSlots)), "l"(rec) : "memory");
                     *reinterpret_cast<volatile unsigned long long *>(&s_items[seq % kItemSlots]) = rec;
@@ -552,9 +552,12 @@ struct PairKernel {
 // stages; big: tiles of up to 256 pair rows
 using Gemm1Small = PairKernel<1, 32, 9, 2>;
 using Gemm2Small = PairKernel<2, 32, 10, 2>;
+using Gemm1Mid = PairKernel<1, 64, 8, 2>;
+using Gemm2Mid = PairKernel<2, 64, 8, 2>;
 using Gemm1Big = PairKernel<1, 128, 6, 2>;
 using Gemm2Big = PairKernel<2, 128, 6, 2>;
 constexpr int kSmallRowsMax = 64;
+constexpr int kMidRowsPerExpert = 100;  // mean slots per candidate (T K / (N + N_Z)) up to which the mid geometry is used
 
 // The small geometry holds at most kSmallRowsMax pair rows of one expert.  Without expert parallelism
 // an expert has at most one pair per token of the call; with it, any number of the received rows.
@@ -564,6 +567,17 @@ bool small_geometry(const zeda_moe *h, const ExpertWork &w) {
 }
 
 }  // namespace
+
+// Mid-sized batches, where an expert holds fewer than about 100 pairs on average and the layer streams
+// every expert's weights once (HBM-bound), get tiles of 128 rows and the ring of eight 24 KB stages:
+// more weight bytes in flight per SM than the six 32 KB stages whose activation half stays half empty.
+// The host knows neither the counts nor the zero share of a call; it goes by the mean number of slots
+// per candidate.
+int tile_rows_for(const zeda_moe *h, int T) {
+    const zeda_moe_config_t &c = h->cfg;
+    if (c.ep_size >= 1) return kPairTileM;
+    return (long long)T * c.top_k <= (long long)kMidRowsPerExpert * (c.n_real + c.n_zero) ? kMidTileM : kPairTileM;
+}
 
 int init_pair_kernels(zeda_moe *h) {
     const zeda_moe_config_t &c = h->cfg;
@@ -592,7 +606,8 @@ int init_pair_kernels(zeda_moe *h) {
         const cuuint32_t box[2] = {kBlockK, (cuuint32_t)(128 >> i)};
         ok = ok && encode_bf16_map(&pm->hmid.m[i], h->ws.hmid, 2, dims, strides, box);
     }
-    ok = ok && Gemm1Small::prepare() && Gemm2Small::prepare() && Gemm1Big::prepare() && Gemm2Big::prepare();
+    ok = ok && Gemm1Small::prepare() && Gemm2Small::prepare() && Gemm1Mid::prepare() && Gemm2Mid::prepare() &&
+         Gemm1Big::prepare() && Gemm2Big::prepare();
     if (!ok) {
         free(pm);
         if (zeda_last_error()[0] == 0) set_error("pair kernel set-up failed: %s", cudaGetErrorString(cudaGetLastError()));
@@ -609,10 +624,11 @@ int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, const E
     const int m_blocks = (c.d_expert + 127) / 128;
     auto go = [&](auto k) {
         return decltype(k)::launch(h, s, pm->w_gate_up, pm->hmid, x, c.d_model, w.counts, w.offsets, w.tile_expert,
-                                   w.tile_row0, w.pair_row, ws.meta, c.d_model, c.d_expert, m_blocks, ws.hmid, c.d_expert);
+                                   w.tile_row0, w.pair_row, ws.meta, c.d_model, c.d_expert, m_blocks, ws.hmid, c.d_expert,
+                                   w.tile_rows);
     };
     // an expert cannot hold more pair rows than the call has tokens (a token selects it at most once)
-    const cudaError_t e = small_geometry(h, w) ? go(Gemm1Small{}) : go(Gemm1Big{});
+    const cudaError_t e = small_geometry(h, w) ? go(Gemm1Small{}) : w.tile_rows == kMidTileM ? go(Gemm1Mid{}) : go(Gemm1Big{});
     return e == cudaSuccess ? 1 : -1;
 }
 
@@ -624,9 +640,9 @@ int launch_experts_gemm2_pair(const zeda_moe *h, const ExpertWork &w, cudaStream
     auto go = [&](auto k) {
         return decltype(k)::launch(h, s, pm->w_down, pm->hmid, (const __nv_bfloat16 *)nullptr, 0, w.counts, w.offsets,
                                    w.tile_expert, w.tile_row0, w.pair_row, ws.meta, c.d_expert, c.d_model, m_blocks,
-                                   ws.obuf, c.d_model);
+                                   ws.obuf, c.d_model, w.tile_rows);
     };
-    const cudaError_t e = small_geometry(h, w) ? go(Gemm2Small{}) : go(Gemm2Big{});
+    const cudaError_t e = small_geometry(h, w) ? go(Gemm2Small{}) : w.tile_rows == kMidTileM ? go(Gemm2Mid{}) : go(Gemm2Big{});
     return e == cudaSuccess ? 1 : -1;
 }
 

@@ -15,21 +15,21 @@ struct ScanShared {
 };
 
 // From per-expert pair counts in sh.cnt: exclusive offsets, P, U, and the tile list of the expert
-// kernels (experts in id order, each with its tiles of kPairTileM rows in row order; the last tile of
+// kernels (experts in id order, each with its tiles of tile_rows rows in row order; the last tile of
 // an expert may be ragged).  Called by every thread of the CTA (blockDim.x >= 32); contains CTA
 // barriers.
 __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, int total_slots,
                                                    int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
                                                    int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
                                                    const WorkLists &wl, bool write_global = true,
-                                                   int list_part = 0, int list_parts = 1) {
+                                                   int list_part = 0, int list_parts = 1, int tile_rows = kPairTileM) {
     if (threadIdx.x < 32) {
         // warp 0 scans the per-expert sequences in steps of 32 with shuffle prefix sums
         int base_off = 0, base_ptile = 0, active = 0, max_rows = 0;
         for (int e0 = 0; e0 < n_real; e0 += 32) {
             const int i = e0 + threadIdx.x;
             const int c = (i < n_real) ? sh.cnt[i] : 0;
-            const int pt = (c + kPairTileM - 1) / kPairTileM;
+            const int pt = (c + tile_rows - 1) / tile_rows;
             int so = c, sp = pt;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -84,7 +84,7 @@ __device__ __forceinline__ void finish_expert_scan(ScanShared &sh, int n_real, i
             if (sh.ptile[mid] <= i) lo = mid; else hi = mid;
         }
         wl.ptile_expert[i] = lo;
-        wl.ptile_row0[i] = (i - sh.ptile[lo]) * kPairTileM;
+        wl.ptile_row0[i] = (i - sh.ptile[lo]) * tile_rows;
     }
 }
 

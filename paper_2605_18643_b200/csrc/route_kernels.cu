@@ -239,7 +239,7 @@ __device__ __forceinline__ void stage_ints(int32_t *__restrict__ dst, const int3
 __global__ void __launch_bounds__(512)
 expert_scan_kernel(int32_t *__restrict__ block_hist, int nblk, int n_real, int total_slots,
                    int32_t *__restrict__ counts, int32_t *__restrict__ offsets,
-                   int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta, const WorkLists wl) {
+                   int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta, const WorkLists wl, int tile_rows) {
     __shared__ ScanShared sh;
     // Exclusive scan of every expert column over the CTA histograms.  The histograms are staged in
     // shared memory slab by slab with independent coalesced loads (a load-scan-store loop straight
@@ -267,7 +267,7 @@ expert_scan_kernel(int32_t *__restrict__ block_hist, int nblk, int n_real, int t
     }
     if (e < n_real) sh.cnt[e] = run;
     __syncthreads();
-    finish_expert_scan(sh, n_real, total_slots, counts, offsets, n_pairs_out, meta, wl);
+    finish_expert_scan(sh, n_real, total_slots, counts, offsets, n_pairs_out, meta, wl, true, 0, 1, tile_rows);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -288,7 +288,7 @@ __global__ void __cluster_dims__(kSmallCluster, 1, 1) __launch_bounds__(kSmallTh
 route_small_kernel(const float *__restrict__ logits, int T, int n_real, int n_cand, int K, int gate_mode,
                    int32_t *__restrict__ topk_idx, float *__restrict__ topk_w, int32_t *__restrict__ counts,
                    int32_t *__restrict__ offsets, int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
-                   const WorkLists wl, int32_t *__restrict__ perm,
+                   const WorkLists wl, int tile_rows, int32_t *__restrict__ perm,
                    int32_t *__restrict__ perm_user, int32_t *__restrict__ inv, int32_t *__restrict__ pair_token) {
     pdl_launch_dependents();
     pdl_wait();
@@ -322,7 +322,7 @@ route_small_kernel(const float *__restrict__ logits, int T, int n_real, int n_ca
         sh.cnt[threadIdx.x] = c;
     }
     __syncthreads();
-    finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, wl);
+    finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, wl, true, 0, 1, tile_rows);
     for (int s = threadIdx.x; s < T * K; s += blockDim.x) {
         const int e = topk_idx[s], tk = s / K;
         int p = -1;
@@ -414,7 +414,7 @@ __global__ void __launch_bounds__(kPlaceWarps * 32)
 slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real, int nblk,
                        const int32_t *__restrict__ block_hist, int32_t *__restrict__ counts,
                        int32_t *__restrict__ offsets, int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
-                       const WorkLists wl, int32_t *__restrict__ perm, int32_t *__restrict__ perm_user,
+                       const WorkLists wl, int tile_rows, int32_t *__restrict__ perm, int32_t *__restrict__ perm_user,
                        int32_t *__restrict__ inv, int32_t *__restrict__ pair_token) {
     pdl_launch_dependents();
     pdl_wait();
@@ -461,7 +461,7 @@ slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n
         }
     }
     __syncthreads();
-    finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, wl, blockIdx.x == 0, blockIdx.x, gridDim.x);
+    finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, wl, blockIdx.x == 0, blockIdx.x, gridDim.x, tile_rows);
     __syncthreads();
     int32_t *mine = pos + warp * n_real;
     const unsigned lt = (1u << lane) - 1u;
@@ -640,6 +640,7 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
     const int nblk = (T + kSortTokens - 1) / kSortTokens;
     int launches = 4;
     const WorkLists wl = {ws.ptile_expert, ws.ptile_row0};
+    const int tile_rows = tile_rows_for(h, T);
 #define ZEDA_RPL_DISPATCH(CALL)                        \
     do {                                               \
         if (n_cand <= 64) { CALL(2); }                 \
@@ -652,7 +653,7 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
 #define ZEDA_CALL_SMALL(R)                                                                                         \
     launch_kernel(h->pdl, route_small_kernel<R>, dim3(kSmallCluster), dim3(kSmallThreads), 0, s,                    \
         logits, T, c.n_real, n_cand, K, c.gate_mode, ws.topk_idx, ws.topk_w, ws.counts, ws.offsets, out.n_pairs,   \
-        ws.meta, wl, ws.perm, out.perm, ws.inv, ws.pair_token)
+        ws.meta, wl, tile_rows, ws.perm, out.perm, ws.inv, ws.pair_token)
         ZEDA_RPL_DISPATCH(ZEDA_CALL_SMALL);
 #undef ZEDA_CALL_SMALL
         launches = 1;
@@ -667,12 +668,12 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
         if (nblk <= kFoldMaxBlocks) {
             launch_kernel(h->pdl, slot_scan_place_kernel, dim3(nblk), dim3(kPlaceWarps * 32),
                           sizeof(int32_t) * ((kPlaceWarps + 1) * c.n_real + kScanSlabInts), s, (const int32_t *)ws.topk_idx, T, K, c.n_real,
-                          nblk, (const int32_t *)ws.block_hist, ws.counts, ws.offsets, out.n_pairs, ws.meta, wl, ws.perm,
+                          nblk, (const int32_t *)ws.block_hist, ws.counts, ws.offsets, out.n_pairs, ws.meta, wl, tile_rows, ws.perm,
                           out.perm, ws.inv, ws.pair_token);
             launches = 3;
         } else {
             expert_scan_kernel<<<1, 512, 0, s>>>(ws.block_hist, nblk, c.n_real, T * K, ws.counts, ws.offsets,
-                                                 out.n_pairs, ws.meta, wl);
+                                                 out.n_pairs, ws.meta, wl, tile_rows);
             slot_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * kPlaceWarps * c.n_real, s>>>(
                 ws.topk_idx, T, K, c.n_real, ws.block_hist, ws.offsets, ws.perm, out.perm, ws.inv, ws.pair_token);
         }
@@ -777,7 +778,7 @@ extern "C" zeda_status_t zeda_compact_static(const int32_t *topk_idx, int32_t T,
     slot_hist_kernel<<<nblk, 256, sizeof(int32_t) * n_real, s>>>(topk_idx, T, top_k, n_real, sc->block_hist);
     const WorkLists wl = {sc->ptile_expert, sc->ptile_row0};
     expert_scan_kernel<<<1, 512, 0, s>>>(sc->block_hist, nblk, n_real, T * top_k, expert_counts, expert_offsets,
-                                         n_pairs, sc->meta, wl);
+                                         n_pairs, sc->meta, wl, kPairTileM);
     slot_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * kPlaceWarps * n_real, s>>>(
         topk_idx, T, top_k, n_real, sc->block_hist, expert_offsets, perm, nullptr, sc->inv, sc->pair_token);
     e = cudaGetLastError();

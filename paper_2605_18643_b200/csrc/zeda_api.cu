@@ -56,7 +56,7 @@ size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int
     const size_t slots = (size_t)c.max_tokens * c.top_k;
     const size_t n_cand = (size_t)c.n_real + c.n_zero;
     const size_t nblk = (c.max_tokens + kSortTokens - 1) / kSortTokens;
-    const size_t tiles = slots / kPairTileM + c.n_real + 1;
+    const size_t tiles = slots / kMidTileM + c.n_real + 1;
     // an expert-parallel handle holds n_local experts and sizes its pair buffers for the rows it may receive
     const bool ep = c.ep_size >= 1;
     const size_t n_local = ep ? (size_t)c.n_real / c.ep_size : (size_t)c.n_real;
@@ -155,7 +155,7 @@ zeda_status_t forward_device(zeda_moe_t *h, const __nv_bfloat16 *x, int T, __nv_
     n += r;
     mark(2);
     const Workspace &ws = h->ws;
-    const ExpertWork work = {ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token, T * h->cfg.top_k};
+    const ExpertWork work = {ws.counts, ws.offsets, ws.ptile_expert, ws.ptile_row0, ws.pair_token, T * h->cfg.top_k, tile_rows_for(h, T)};
     r = launch_experts_gemm1_pair(h, x, work, s);
     if (r < 0) return cuda_fail("expert GEMM1 launch", cudaGetLastError());
     n += r;
@@ -364,7 +364,7 @@ zeda_status_t zeda_ep_experts(zeda_moe_t *h, const void *recv_rows, const int32_
     int n = launch_ep_plan(h, recv_counts, n_rows, s);
     if (n < 0) return cuda_fail("plan launch", cudaGetLastError());
     const Workspace &ws = h->ws;
-    const ExpertWork work = {ws.ep_counts, ws.ep_offsets, ws.ep_tile_expert, ws.ep_tile_row0, ws.ep_pair_row, n_rows};
+    const ExpertWork work = {ws.ep_counts, ws.ep_offsets, ws.ep_tile_expert, ws.ep_tile_row0, ws.ep_pair_row, n_rows, kPairTileM};
     int r = launch_experts_gemm1_pair(h, static_cast<const __nv_bfloat16 *>(recv_rows), work, s);
     if (r < 0) return cuda_fail("expert GEMM1 launch", cudaGetLastError());
     n += r;

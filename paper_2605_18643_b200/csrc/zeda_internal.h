@@ -12,7 +12,8 @@ namespace zeda {
 constexpr int kMaxCand = 512;       // N + N_Z limit (16 logits per lane in the top-K warp)
 constexpr int kMaxTopK = 16;
 constexpr int kSortTokens = 128;    // tokens per CTA in the counting sort (histogram / placement)
-constexpr int kPairTileM = 256;     // pair rows per tile of the expert kernels (one CTA pair, N <= 256)
+constexpr int kPairTileM = 256;     // most pair rows per tile of the expert kernels (one CTA pair, N <= 256)
+constexpr int kMidTileM = 128;      // tile rows of the geometry for mid-sized batches
 constexpr int kMaxEpRanks = 64;     // expert-parallel group size limit
 
 // Device-resident counters of one call.
@@ -61,6 +62,7 @@ struct Workspace {
 struct ExpertWork {
     const int32_t *counts, *offsets, *tile_expert, *tile_row0, *pair_row;
     int rows_bound;  // upper bound of the pair rows of a call (host-side; picks the kernel geometry)
+    int tile_rows;   // pair rows per tile of the tile list (kPairTileM or kMidTileM)
 };
 
 // Device-side tile list written by the expert scan: experts in id order, each with its tiles of at
@@ -126,6 +128,9 @@ inline long long router_part_rows(long long max_tokens) {
 int router_split_factor(const zeda_moe *h, int T);
 int launch_router_logits_tile(const zeda_moe *h, const __nv_bfloat16 *x, int T, float *logits, int split, cudaStream_t s);
 int init_pair_kernels(zeda_moe *h);
+// Pair rows per tile for a call of T tokens on this handle: the routing pass builds the tile list with
+// it and the expert kernels of the same call are picked to match.
+int tile_rows_for(const zeda_moe *h, int T);
 int launch_token_zero_share(const zeda_moe *h, int T, float *out, cudaStream_t s);
 int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, const ExpertWork &w, cudaStream_t s);
 int launch_experts_gemm2_pair(const zeda_moe *h, const ExpertWork &w, cudaStream_t s);
