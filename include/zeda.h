@@ -143,9 +143,18 @@ zeda_status_t zeda_router_logits(zeda_moe_t *h, const void *x, int32_t T, float 
 zeda_status_t zeda_moe_forward(zeda_moe_t *h, const void *x, int32_t T, void *y, void *stream);
 
 /* The same forward for callers whose activations live in HOST memory: copies x to the device,
- * runs the layer, copies y back, all on `stream`, and synchronises the stream before returning.
+ * runs the layer, copies y back, and returns once y_host is complete (it synchronises `stream`).
  *   x_host  host [T, d_model] bf16     y_host  host [T, d_model] bf16
- * Pinned host memory makes the copies asynchronous; pageable memory works but is slower. */
+ * Pinned host memory makes the copies asynchronous; pageable memory works but is slower.
+ * Batches of 4096 tokens or more are processed as two chunks (the layer is per token): the device
+ * work of both stays on `stream`, the copies run on two streams that the handle creates on first use
+ * (host objects; no device memory), so the second chunk is copied in while the first is computed and
+ * the first is copied back while the second is computed.  The result is, bit for bit, that of
+ * zeda_moe_forward on the two chunks (the first (T/2 rounded up to a multiple of 256) tokens, then the
+ * rest); against one call on the whole batch the routing weights can differ in their last bits,
+ * because the router slices its reduction axis by batch size.  Afterwards the routing kept in the
+ * handle (statistics, counters) is that of the second chunk, except the launch count, which covers
+ * both. */
 zeda_status_t zeda_moe_forward_host(zeda_moe_t *h, const void *x_host, int32_t T, void *y_host,
                                     void *stream);
 

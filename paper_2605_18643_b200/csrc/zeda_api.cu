@@ -238,6 +238,8 @@ zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_
     h->profiling = false;
     h->profiled_last = false;
     for (auto &ev : h->ev) ev = nullptr;
+    h->copy_in = h->copy_out = nullptr;
+    for (auto &ev : h->ev_host) ev = nullptr;
     carve(*cfg, static_cast<unsigned char *>(workspace), &h->ws, &h->max_tiles);
     if (init_route_kernels(h) < 0) { delete h; return cuda_fail("kernel set-up", cudaGetLastError()); }
     if (init_pair_kernels(h) < 0) { delete h; return ZEDA_ERR_CUDA; }
@@ -300,6 +302,11 @@ zeda_status_t zeda_moe_forward(zeda_moe_t *h, const void *x, int32_t T, void *y,
                           static_cast<cudaStream_t>(stream));
 }
 
+// Batches of at least this many tokens go through the host-buffer entry point in two chunks, so that
+// the copy of the second chunk runs under the layer of the first and the copy back of the first under
+// the layer of the second.
+static const int kHostSplitMinTokens = 4096;
+
 zeda_status_t zeda_moe_forward_host(zeda_moe_t *h, const void *x_host, int32_t T, void *y_host, void *stream) {
     if (!h) { set_error("handle is NULL"); return ZEDA_ERR_INVALID_ARG; }
     if (T < 0 || T > h->cfg.max_tokens) { set_error("T=%d outside [0, max_tokens=%d]", T, h->cfg.max_tokens); return ZEDA_ERR_INVALID_ARG; }
@@ -309,14 +316,57 @@ zeda_status_t zeda_moe_forward_host(zeda_moe_t *h, const void *x_host, int32_t T
     cudaError_t e = cudaSetDevice(h->cfg.device);
     if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t bytes = (size_t)T * h->cfg.d_model * 2;
-    e = cudaMemcpyAsync(h->ws.x_stage, x_host, bytes, cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return cuda_fail("copy of x to the device", e);
-    zeda_status_t st = forward_device(h, h->ws.x_stage, T, h->ws.y_stage, s);
+    const size_t row = (size_t)h->cfg.d_model * 2;
+    if (T < kHostSplitMinTokens) {
+        e = cudaMemcpyAsync(h->ws.x_stage, x_host, T * row, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return cuda_fail("copy of x to the device", e);
+        zeda_status_t st = forward_device(h, h->ws.x_stage, T, h->ws.y_stage, s);
+        if (st != ZEDA_OK) return st;
+        e = cudaMemcpyAsync(y_host, h->ws.y_stage, T * row, cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return cuda_fail("copy of y to the host", e);
+        e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
+        return ZEDA_OK;
+    }
+    // Two chunks.  The layer is per token (Eq. 1), so the chunks are two independent calls; their device
+    // work stays on `stream`, one after the other (they share the workspace), the copies run on two
+    // streams of the handle.
+    if (!h->copy_in) {
+        e = cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking);
+        for (auto &ev : h->ev_host)
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+        if (e != cudaSuccess) return cuda_fail("stream / event creation", e);
+    }
+    const int T0 = (T / 2 + 255) / 256 * 256, T1 = T - T0;
+    const char *xh = static_cast<const char *>(x_host);
+    char *yh = static_cast<char *>(y_host);
+    __nv_bfloat16 *xs = h->ws.x_stage, *ys = h->ws.y_stage;
+    cudaEvent_t *ev = h->ev_host;  // 0 start, 1-2 chunk copied in, 3-4 chunk computed, 5 all copied out
+    bool ok = cudaEventRecord(ev[0], s) == cudaSuccess && cudaStreamWaitEvent(h->copy_in, ev[0], 0) == cudaSuccess &&
+              cudaStreamWaitEvent(h->copy_out, ev[0], 0) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(xs, xh, T0 * row, cudaMemcpyHostToDevice, h->copy_in) == cudaSuccess &&
+         cudaEventRecord(ev[1], h->copy_in) == cudaSuccess &&
+         cudaMemcpyAsync(xs + (size_t)T0 * h->cfg.d_model, xh + T0 * row, T1 * row, cudaMemcpyHostToDevice, h->copy_in) == cudaSuccess &&
+         cudaEventRecord(ev[2], h->copy_in) == cudaSuccess;
+    if (!ok) return cuda_fail("copy of x to the device", cudaGetLastError());
+    if (cudaStreamWaitEvent(s, ev[1], 0) != cudaSuccess) return cuda_fail("cudaStreamWaitEvent", cudaGetLastError());
+    zeda_status_t st = forward_device(h, xs, T0, ys, s);
     if (st != ZEDA_OK) return st;
-    e = cudaMemcpyAsync(y_host, h->ws.y_stage, bytes, cudaMemcpyDeviceToHost, s);
-    if (e != cudaSuccess) return cuda_fail("copy of y to the host", e);
-    e = cudaStreamSynchronize(s);
+    if (cudaEventRecord(ev[3], s) != cudaSuccess || cudaStreamWaitEvent(s, ev[2], 0) != cudaSuccess)
+        return cuda_fail("cudaEventRecord", cudaGetLastError());
+    const int launches0 = h->last_launches;
+    st = forward_device(h, xs + (size_t)T0 * h->cfg.d_model, T1, ys + (size_t)T0 * h->cfg.d_model, s);
+    if (st != ZEDA_OK) return st;
+    h->last_launches += launches0;
+    ok = cudaEventRecord(ev[4], s) == cudaSuccess && cudaStreamWaitEvent(h->copy_out, ev[3], 0) == cudaSuccess &&
+         cudaMemcpyAsync(yh, ys, T0 * row, cudaMemcpyDeviceToHost, h->copy_out) == cudaSuccess &&
+         cudaStreamWaitEvent(h->copy_out, ev[4], 0) == cudaSuccess &&
+         cudaMemcpyAsync(yh + T0 * row, ys + (size_t)T0 * h->cfg.d_model, T1 * row, cudaMemcpyDeviceToHost, h->copy_out) == cudaSuccess &&
+         cudaEventRecord(ev[5], h->copy_out) == cudaSuccess;
+    if (!ok) return cuda_fail("copy of y to the host", cudaGetLastError());
+    e = cudaEventSynchronize(ev[5]);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail("cudaStreamSynchronize", e);
     return ZEDA_OK;
 }
@@ -496,6 +546,9 @@ zeda_status_t zeda_moe_destroy(zeda_moe_t *h) {
         else if (err != 0) { set_error(kDeviceFailure, err); st = ZEDA_ERR_TIMEOUT; }
     }
     for (auto &ev : h->ev) if (ev) cudaEventDestroy(ev);
+    for (auto &ev : h->ev_host) if (ev) cudaEventDestroy(ev);
+    if (h->copy_in) cudaStreamDestroy(h->copy_in);
+    if (h->copy_out) cudaStreamDestroy(h->copy_out);
     if (h->pmaps) free(h->pmaps);
     if (h->router_maps) free(h->router_maps);
     delete h;

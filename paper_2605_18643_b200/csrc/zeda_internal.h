@@ -101,6 +101,9 @@ struct zeda_moe {
     bool profiled_last;
     int last_routed_tokens;  // T of the most recent routing pass on this handle
     cudaEvent_t ev[ZEDA_STAGE_COUNT + 1];
+    // host-buffer entry point: copy streams and events of its two-chunk pipeline (made on first use)
+    cudaStream_t copy_in, copy_out;
+    cudaEvent_t ev_host[6];
 };
 
 namespace zeda {

@@ -225,6 +225,29 @@ def test_host_buffer_entry_point(zeda):
     m.close()
 
 
+def test_host_buffer_entry_point_in_two_chunks(zeda):
+    # from 4096 tokens on the host-buffer call copies and computes in two chunks on three streams: the
+    # result is, bit for bit, that of the two chunks passed through zeda_moe_forward one after the other
+    # (also for a ragged split and on a second call), and the whole-batch result up to the last bits of
+    # the routing weights (the router slices its reduction axis by batch size)
+    for T in (4096, 5000):
+        wl = inputs.tiny(seed=17, T=T)
+        dev = torch.device("cuda:0")
+        m = zeda.from_workload(wl, dev)
+        x = wl.x.to(dev)
+        T0 = (T // 2 + 255) // 256 * 256
+        y_whole = m.forward(x).float().cpu()
+        y_chunks = torch.cat([m.forward(x[:T0].contiguous()), m.forward(x[T0:].contiguous())]).cpu()
+        x_pin = wl.x.pin_memory()
+        for _ in range(2):
+            y_host = m.forward_host(x_pin)
+            assert torch.equal(y_chunks.view(torch.int16), y_host.view(torch.int16))
+        assert m.last_counters()[3] > 0
+        diff = (y_host.float() - y_whole).norm() / y_whole.norm()
+        assert float(diff) < 1e-3
+        m.close()
+
+
 def test_routing_statistics(zeda):
     wl = inputs.tiny(seed=9, T=200)
     dev = torch.device("cuda:0")
