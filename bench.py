@@ -300,15 +300,22 @@ def run_stack(args, peaks, peaks_kind, dev, world, rank, barrier, dist):
         r0 = inputs.replica_tokens(layers[0], rank)
     r_init = r0.to(dev)
     r = r_init.clone()
-    h = torch.empty_like(r)
-    ys = [torch.empty_like(r), torch.empty_like(r)]
+    hs = [torch.empty_like(r), torch.empty_like(r)]
+    y_last = torch.empty_like(r)
+    fused = args.stack_glue == "fused"
 
     def one_pass():
         r.copy_(r_init)
+        if fused:
+            # the glue of layers 1.. rides in the last pass of the layer before it
+            zeda.residual_rmsnorm(r, None, hs[0])
+            for l, m in enumerate(mods[:-1]):
+                m.forward_residual(hs[l & 1], r, hs[(l + 1) & 1])
+            return mods[-1].forward(hs[(len(mods) - 1) & 1], y_last)
         y = None
         for l, m in enumerate(mods):
-            zeda.residual_rmsnorm(r, y, h)
-            y = m.forward(h, ys[l & 1])
+            zeda.residual_rmsnorm(r, y, hs[0])
+            y = m.forward(hs[0], y_last if l & 1 else hs[1])
         return y
 
     clocks = ClockSampler(dev.index or 0)
@@ -378,7 +385,7 @@ def run_stack(args, peaks, peaks_kind, dev, world, rank, barrier, dist):
             "metric": METRIC, "value": job_tokens_per_s(world, T, ms_per_step), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "stack", "layers": len(mods), "T": T, "d": d, "d_expert": He, "n_real": E,
+            "config": {"workload": "stack", "layers": len(mods), "glue": args.stack_glue, "T": T, "d": d, "d_expert": He, "n_real": E,
                        "n_zero": Z, "top_k": K, "seed": 0, "pairs_per_layer_min_max": [min(Ps), max(Ps)],
                        "zero_slot_fraction_mean": round(1.0 - sum(Ps) / (len(Ps) * T * K), 4),
                        "weights_gb": round(len(mods) * E * 3 * d * He * 2 / 1e9, 2),
@@ -387,7 +394,7 @@ def run_stack(args, peaks, peaks_kind, dev, world, rank, barrier, dist):
             "clocks": clock_info,
             "e2e": {"value": world * T * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": T * d * 2,
                     "d2h_bytes_per_step": T * d * 2, "ms_per_step": 1e3 * e2e_s / args.steps},
-            "gpu_launches": (sum(c[3] for c in counters) + len(mods)) * args.steps,
+            "gpu_launches": (sum(c[3] for c in counters) + (1 if fused else len(mods))) * args.steps,
             "roofline": roof,
             "layer_roofline": {"t_roof_us": t_roof * 1e6, "frac": t_roof / (ms_per_step * 1e-3),
                                "t_roof_us_sustained": t_roof_s * 1e6,
@@ -615,6 +622,8 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="prefill only: skip the nested zero-fraction sweep")
     ap.add_argument("--layers", type=int, default=48, help="layers of --workload stack")
     ap.add_argument("--stack-tokens", type=int, default=4096, help="tokens per pass of --workload stack")
+    ap.add_argument("--stack-glue", choices=["fused", "separate"], default="fused",
+                    help="--workload stack: residual + RMSNorm fused into each layer's combine pass, or its own kernel")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

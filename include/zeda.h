@@ -168,6 +168,21 @@ zeda_status_t zeda_moe_forward_host(zeda_moe_t *h, const void *x_host, int32_t T
 zeda_status_t zeda_residual_rmsnorm(void *r, const void *y, void *h, int32_t T, int32_t d_model, float eps,
                                     void *stream);
 
+/* One layer of a stack with the glue fused into its last pass (same layer as zeda_moe_forward, Eq. 1;
+ * same glue as zeda_residual_rmsnorm): the layer output y~ is not stored, instead
+ *   r      <- bf16(r + bf16(y~(x)))          residual stream, updated in place
+ *   h_next  = r / sqrt(mean(r^2) + eps)      the next layer's input
+ * The results are, bit for bit, those of zeda_moe_forward(h, x, T, y) followed by
+ * zeda_residual_rmsnorm(r, y, h_next, T, d_model, eps): one launch and one round trip of y through
+ * device memory fewer per layer.
+ *   x  dev [T, d_model] bf16 (this layer's input)   r  dev [T, d_model] bf16 (in/out)
+ *   h_next  dev [T, d_model] bf16 (out)
+ * x, r and h_next must not overlap one another (ZEDA_ERR_INVALID_ARG).  d_model <= 2048 (a token's
+ * row is held by one thread block), otherwise ZEDA_ERR_UNSUPPORTED: use the two calls.  Other
+ * arguments, errors and the routing kept in the handle as for zeda_moe_forward. */
+zeda_status_t zeda_moe_forward_residual(zeda_moe_t *h, const void *x, int32_t T, void *r, void *h_next, float eps,
+                                        void *stream);
+
 /* Routing statistics of the most recent zeda_route / zeda_moe_forward call on this handle
  * (Section 2.2, Eq. 4-6), computed on the device from that call's routing:
  *   f      dev [N+N_Z] fp32  share of tokens whose top-K set holds candidate i (f_i), or NULL

@@ -140,7 +140,10 @@ int route_into(zeda_moe_t *h, const __nv_bfloat16 *x, const float *logits_in, in
     return n + r;
 }
 
-zeda_status_t forward_device(zeda_moe_t *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s) {
+// With resid given, the call ends in the fused combine + glue pass: resid <- bf16(resid + y) and
+// the normalised residual goes where y would have gone.
+zeda_status_t forward_device(zeda_moe_t *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s,
+                             __nv_bfloat16 *resid = nullptr, float eps = 0.f) {
     const bool prof = h->profiling;
     auto mark = [&](int i) { if (prof) cudaEventRecord(h->ev[i], s); };
     mark(0);
@@ -164,7 +167,7 @@ zeda_status_t forward_device(zeda_moe_t *h, const __nv_bfloat16 *x, int T, __nv_
     if (r < 0) return cuda_fail("expert GEMM2 launch", cudaGetLastError());
     n += r;
     mark(4);
-    r = launch_combine(h, x, T, y, s);
+    r = resid ? launch_combine_glue(h, x, T, resid, y, eps, s) : launch_combine(h, x, T, y, s);
     if (r < 0) return cuda_fail("combine launch", cudaGetLastError());
     mark(5);
     h->profiled_last = prof;
@@ -300,6 +303,23 @@ zeda_status_t zeda_moe_forward(zeda_moe_t *h, const void *x, int32_t T, void *y,
     if (xb < yb + bytes && yb < xb + bytes) { set_error("x and y overlap"); return ZEDA_ERR_INVALID_ARG; }
     return forward_device(h, static_cast<const __nv_bfloat16 *>(x), T, static_cast<__nv_bfloat16 *>(y),
                           static_cast<cudaStream_t>(stream));
+}
+
+zeda_status_t zeda_moe_forward_residual(zeda_moe_t *h, const void *x, int32_t T, void *r, void *h_next, float eps,
+                                        void *stream) {
+    zeda_status_t st = check_call(h, x, T, "x");
+    if (st != ZEDA_OK || T == 0) return st;
+    if (h->cfg.ep_size >= 1) { set_error("an expert-parallel handle (ep_size >= 1) runs the layer through the zeda_ep_* calls"); return ZEDA_ERR_INVALID_ARG; }
+    if (!combine_glue_supported(h)) { set_error("the fused residual form needs d_model <= 2048"); return ZEDA_ERR_UNSUPPORTED; }
+    if (!r || !h_next || !aligned16(r) || !aligned16(h_next)) { set_error("r or h_next is NULL or not 16-byte aligned"); return ZEDA_ERR_INVALID_ARG; }
+    if (!(eps >= 0.f)) { set_error("eps must be >= 0"); return ZEDA_ERR_INVALID_ARG; }
+    const size_t bytes = (size_t)T * h->cfg.d_model * 2;
+    const char *b[3] = {static_cast<const char *>(x), static_cast<const char *>(r), static_cast<const char *>(h_next)};
+    for (int i = 0; i < 3; ++i)
+        for (int j = i + 1; j < 3; ++j)
+            if (b[i] < b[j] + bytes && b[j] < b[i] + bytes) { set_error("x, r and h_next overlap"); return ZEDA_ERR_INVALID_ARG; }
+    return forward_device(h, static_cast<const __nv_bfloat16 *>(x), T, static_cast<__nv_bfloat16 *>(h_next),
+                          static_cast<cudaStream_t>(stream), static_cast<__nv_bfloat16 *>(r), eps);
 }
 
 // Batches of at least this many tokens go through the host-buffer entry point in two chunks, so that

@@ -146,6 +146,10 @@ int launch_combine_rows(const zeda_moe *h, const __nv_bfloat16 *rows, const __nv
                         cudaStream_t s);
 int launch_wait_selftest(const zeda_moe *h, long long limit_cycles, cudaStream_t s);
 int launch_combine(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *y, cudaStream_t s);
+// combine fused with the residual + RMSNorm glue of a layer stack (rows of up to 2048 elements)
+bool combine_glue_supported(const zeda_moe *h);
+int launch_combine_glue(const zeda_moe *h, const __nv_bfloat16 *x, int T, __nv_bfloat16 *resid, __nv_bfloat16 *h_next, float eps,
+                        cudaStream_t s);
 
 void set_error(const char *fmt, ...);
 // remembers the error of a failed kernel launch for the status message of the API call (the runtime's

@@ -23,7 +23,7 @@ FLAG_NONE, FLAG_NO_DEPENDENT_LAUNCH = 0, 4
 
 EXPORTS = (
     "zeda_moe_workspace_bytes", "zeda_moe_create", "zeda_route", "zeda_route_from_logits",
-    "zeda_router_logits", "zeda_moe_forward", "zeda_moe_forward_host", "zeda_moe_stats",
+    "zeda_router_logits", "zeda_moe_forward", "zeda_moe_forward_residual", "zeda_moe_forward_host", "zeda_moe_stats",
     "zeda_moe_token_zero_share", "zeda_moe_last_counters", "zeda_moe_set_profiling", "zeda_moe_stage_ms", "zeda_residual_rmsnorm",
     "zeda_moe_selftest_wait", "zeda_moe_clear_error",
     "zeda_ep_dispatch", "zeda_ep_experts", "zeda_ep_combine",
@@ -80,6 +80,8 @@ def _load() -> ctypes.CDLL:
     lib.zeda_moe_clear_error.argtypes = [vp, vp]
     lib.zeda_residual_rmsnorm.restype = i32
     lib.zeda_residual_rmsnorm.argtypes = [vp, vp, vp, i32, i32, ctypes.c_float, vp]
+    lib.zeda_moe_forward_residual.restype = i32
+    lib.zeda_moe_forward_residual.argtypes = [vp, vp, i32, vp, vp, ctypes.c_float, vp]
     lib.zeda_ep_dispatch.restype = i32
     lib.zeda_ep_dispatch.argtypes = [vp, vp, i32, vp, vp, vp, vp]
     lib.zeda_ep_experts.restype = i32
@@ -237,6 +239,16 @@ class ZedaMoE:
             out = torch.empty_like(x)
         _check(lib.zeda_moe_forward(self._h, _ptr(x), T, _ptr(out), _stream(self.device)))
         return out
+
+    def forward_residual(self, x: torch.Tensor, r: torch.Tensor, h_next: torch.Tensor, eps: float = 1e-6) -> torch.Tensor:
+        """zeda_moe_forward_residual: the layer on x with the stack glue fused into its last pass
+        (r <- r + y in place, h_next = RMSNorm(r)); asynchronous on the current stream."""
+        T = self._check_x(x)
+        for t in (r, h_next):
+            assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and t.shape == x.shape
+        _check(lib.zeda_moe_forward_residual(self._h, _ptr(x), T, _ptr(r), _ptr(h_next), float(eps),
+                                             _stream(self.device)))
+        return h_next
 
     def forward_host(self, x_host: torch.Tensor, out_host: Optional[torch.Tensor] = None) -> torch.Tensor:
         """zeda_moe_forward_host on CPU tensors (pinned preferred); returns after the copy back."""

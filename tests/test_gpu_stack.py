@@ -55,6 +55,54 @@ def test_residual_rmsnorm_argument_errors(zeda):
     zeda.residual_rmsnorm(torch.zeros(0, 64, dtype=torch.bfloat16, device=dev), None)  # empty: nothing happens
 
 
+@pytest.mark.parametrize("T,d,kind", [(300, 256, "zero"), (1, 64, "zero"), (777, 2048, "zero"), (300, 448, "copy"),
+                                      (64, 1024, "copy")])
+def test_fused_residual_form_gives_the_bits_of_the_two_calls(zeda, T, d, kind):
+    # zeda_moe_forward_residual against zeda_moe_forward + zeda_residual_rmsnorm on the same inputs:
+    # the residual stream and the next layer's input must be the same bits (the fused pass rounds
+    # y to bf16 before the addition and adds the squares in the glue kernel's order).  The two-call
+    # form itself is held against the oracle by the tests below.
+    He, E, Z, K = 128, 8, 4, 3
+    dev = torch.device("cuda:0")
+    wl = inputs.make_layer("fused", T=T, d=d, He=He, E=E, Z=Z, K=K, seed=77, zero_fraction=0.5)
+    m = zeda.from_workload(wl, dev, expert_kind=zeda.EXPERT_COPY if kind == "copy" else zeda.EXPERT_ZERO)
+    r0 = inputs.make_layer("fused_r", T=T, d=d, He=He, E=E, Z=Z, K=K, seed=78).x.to(dev)
+    x = zeda.residual_rmsnorm(r0.clone(), None)
+    # two calls
+    r_a = r0.clone()
+    y = m.forward(x)
+    h_a = zeda.residual_rmsnorm(r_a, y, eps=1e-5)
+    # fused
+    r_b = r0.clone()
+    h_b = torch.full_like(r0, float("nan"))
+    m.forward_residual(x, r_b, h_b, eps=1e-5)
+    torch.cuda.synchronize()
+    assert torch.any(y != 0)
+    assert np.array_equal(_bits(r_a), _bits(r_b))
+    assert np.array_equal(_bits(h_a), _bits(h_b))
+    # argument errors: overlapping buffers, missing pointers
+    with pytest.raises(zeda.ZedaError):
+        m.forward_residual(x, r_b, r_b)
+    with pytest.raises(zeda.ZedaError):
+        m.forward_residual(x, x.clone(), x)
+    m.close()
+
+
+def test_fused_residual_form_refuses_rows_wider_than_one_block(zeda):
+    T, d, He, E, Z, K = 16, 2112, 64, 4, 2, 2
+    dev = torch.device("cuda:0")
+    wl = inputs.make_layer("wide", T=T, d=d, He=He, E=E, Z=Z, K=K, seed=5)
+    m = zeda.from_workload(wl, dev)
+    x = wl.x.to(dev)
+    with pytest.raises(zeda.ZedaError) as ei:
+        m.forward_residual(x, x.clone(), torch.empty_like(x))
+    assert ei.value.status == zeda.ERR_UNSUPPORTED
+    y = m.forward(x)  # the two-call form still serves such rows
+    zeda.residual_rmsnorm(x.clone(), y)
+    torch.cuda.synchronize()
+    m.close()
+
+
 def test_three_layer_stack_per_layer_parity(zeda):
     T, d, He, E, Z, K = 300, 256, 128, 8, 4, 2
     dev = torch.device("cuda:0")
