@@ -20,7 +20,8 @@
 // One CTA per SM, persistent over a device-side work list (the host never learns P or the counts).
 // Warp 0: TMA producer (weights).  Warp 1: TMEM allocation, and in the leader CTA the MMA issue.
 // Warp 2 (GEMM1): gather relay.  Warp 3 (GEMM2): TMA producer of the Hmid rows.  Warps 4-7:
-// epilogue.  Warps 8-11 (GEMM1): x-row gather.  Full barriers live in the leader CTA and count the
+// epilogue.  Warps 8-11 (GEMM1): x-row gather.  One more warp per TMA stream (GEMM1: warp 12; GEMM2:
+// warps 8 and 9) takes every second k-step.  Full barriers live in the leader CTA and count the
 // TMA bytes (and gather relays) of both CTAs; stage-empty and accumulator-full barriers are
 // signalled in both CTAs by multicast commits.  The issuing warps (TMA producers, MMA issue, relay)
 // run their loops with all 32 lanes converged: every lane waits on the barrier, one elected lane
@@ -42,8 +43,9 @@ constexpr int kBlockK = 64;                     // bf16 elements per k-step = on
 constexpr int kATileBytes = 128 * kBlockK * 2;  // 16 KB: this CTA's 128 weight rows of one k-step
 constexpr int kRowBytes = kBlockK * 2;          // 128
 constexpr int kAccCols = 256;                   // TMEM columns of one accumulator buffer
-constexpr int kThreads = 256;                   // GEMM2
-constexpr int kThreadsGather = 384;             // GEMM1: + four gather warps
+constexpr int kThreads = 320;                   // GEMM2: warps 8, 9 are the second issuers of the two TMA streams
+constexpr int kThreadsGather = 416;             // GEMM1: four gather warps, warp 12 the second weight issuer
+constexpr int kProducers = 2;                   // warps that share a TMA stream, k-step c going to warp c mod 2
 constexpr int kPatchBytes = 4 * 32 * 32 * 2;    // per epilogue warp: [32 pair rows][32 features] bf16, for 16-byte stores
 constexpr int kXchgBytes = 2 * 2 * 32 * 32 * 4; // GEMM1 gate/up swap: [warp pair][direction][32 cols][32 lanes] fp32
 
@@ -61,6 +63,14 @@ struct PairMaps {
 
 struct Item {
     int e, pos0, n, mb;
+};
+
+// one k-step of an item in the ring: the weight tile(s), then this CTA's pair rows
+template <int HALF_MAX, int DBL_ROWS>
+struct StageBytes {
+    static constexpr int kSingle = kATileBytes + HALF_MAX * kRowBytes;
+    static constexpr int kDouble = DBL_ROWS > 0 ? 2 * kATileBytes + (DBL_ROWS / 2) * kRowBytes : 0;
+    static constexpr int value = kSingle > kDouble ? kSingle : kDouble;
 };
 
 __device__ __forceinline__ Item load_item(long long item, int m_blocks, int tile_rows, const int32_t *tile_expert,
@@ -134,14 +144,23 @@ __device__ __forceinline__ void named_sync(int id, int threads) {
 
 __device__ __forceinline__ float swiglu(float g, float u) { return __fdividef(g * u, 1.f + __expf(-g)); }
 
+// A tile of at most DBL_ROWS pair rows takes two blocks of weight rows per item ("double item"): a
+// k-step of such a tile costs the pipeline the same time whether it carries one block or two (the
+// tensor pipe is idle most of it: an MMA of N <= 128 columns takes about 70 cycles however narrow it
+// is, and the rest is the barrier round trips of the stage), so a double item moves an expert's weights
+// through the SM pair twice as fast.  Its two accumulators share one TMEM buffer (columns 0.. and
+// 128..), its stage holds both weight tiles and the pair rows: 16 + 16 + DBL_ROWS / 2 * 128 bytes.
+__device__ __forceinline__ bool double_item(int dbl_rows, int n, int mb, int m_blocks) {
+    return n <= dbl_rows && !(mb & 1) && mb + 1 < m_blocks;
+}
+
 // MODE 1: GEMM1 + SwiGLU -> Hmid[pos, f].   MODE 2: GEMM2 -> O[pos, row].
 // HALF_MAX: most B rows one CTA loads per k-step (the tile's column count is at most 2 * HALF_MAX).
-// ACC_BUFS: accumulator buffers in TMEM.  2: one CTA per SM, the epilogue of a tile runs under the MMAs
-// of the CTA's next tile.  1: the CTA takes half of the SM (256 TMEM columns, at most half of the
-// shared memory), two CTAs of different pairs share an SM and fill each other's gaps (epilogues, tiles
-// of few rows that wait on their weight stream).
-template <int MODE, int HALF_MAX, int STAGES, int ACC_BUFS>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MODE == 1 ? kThreadsGather : kThreads, ACC_BUFS == 1 ? 2 : 1)
+// DBL_ROWS: tiles of at most this many pair rows run as double items (0: none; at most 128).
+// One CTA per SM with two accumulator buffers in TMEM: the epilogue of a tile runs under the MMAs of
+// the CTA's next tile.
+template <int MODE, int HALF_MAX, int STAGES, int DBL_ROWS>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(MODE == 1 ? kThreadsGather : kThreads, 1)
 expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ RowMaps maps_b,
                         const __nv_bfloat16 *__restrict__ x, int x_ld, const int32_t *__restrict__ counts,
                         const int32_t *__restrict__ offsets, const int32_t *__restrict__ tile_expert,
@@ -149,8 +168,9 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                         int32_t *__restrict__ meta, int kdim, int out_rows, int m_blocks,
                         __nv_bfloat16 *__restrict__ out, int out_ld, int tile_rows) {
     static_assert(STAGES <= 10, "the item queue's depth assumes at most 10 ring stages");
-    constexpr int kStageBytes = kATileBytes + HALF_MAX * kRowBytes;
-    constexpr int kTmemCols = ACC_BUFS * kAccCols;
+    static_assert(DBL_ROWS <= 128 && DBL_ROWS % 32 == 0 && DBL_ROWS <= 2 * HALF_MAX, "two accumulators of a double item share 256 columns");
+    constexpr int kStageBytes = StageBytes<HALF_MAX, DBL_ROWS>::value;
+    constexpr int kTmemCols = 2 * kAccCols;
     pdl_launch_dependents();
     extern __shared__ __align__(1024) unsigned char pair_smem[];
     __shared__ __align__(8) unsigned long long bars[3 * STAGES + 4];
@@ -202,8 +222,12 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     const uint32_t full0 = mapa(bar_full, 0);      // the leader's full barriers, as seen from either CTA
     const uint32_t tempty0 = mapa(bar_tempty, 0);  // the leader's accumulator-free barriers
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer (weights)
+    const int w_prod = warp == 0 ? 0 : (warp == (MODE == 1 ? 12 : 8) ? 1 : -1);
+    const int b_prod = MODE == 2 ? (warp == 3 ? 0 : (warp == 9 ? 1 : -1)) : -1;
+    if (w_prod >= 0) {
+        // ------------------------------------------------------------------ TMA producers (weights)
+        // Issuing one tensor copy keeps a warp busy for several hundred cycles; two warps take the
+        // k-steps in turn.
         {
             uint32_t it_count = 0;
             bool ok = true;
@@ -211,10 +235,12 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 Item it;
                 const int got = next_item(queue, seq, it, abort_flag);
                 if (got <= 0) { ok = got == 0; break; }
-                if (lane == 0) *reinterpret_cast<volatile int *>(&s_prod_seq) = (int)seq;  // read by the scheduler warp
+                if (w_prod == 0 && lane == 0) *reinterpret_cast<volatile int *>(&s_prod_seq) = (int)seq;  // read by the scheduler warp
                 const int half = ((it.n + 31) >> 5) << 4;  // B rows of this CTA; the tile has 2 * half columns
-                const uint32_t bytes = 2u * (uint32_t)(kATileBytes + (MODE == 2 ? half * kRowBytes : 0));
+                const bool dbl = double_item(DBL_ROWS, it.n, it.mb, m_blocks);
+                const uint32_t bytes = 2u * (uint32_t)((dbl ? 2 : 1) * kATileBytes + (MODE == 2 ? half * kRowBytes : 0));
                 for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
+                    if ((int)(it_count % kProducers) != w_prod) continue;
                     const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
                     ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag));
                     if (!ok) break;
@@ -226,6 +252,12 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                             tma_load_5d_pair(sa, &map_a, ks * kBlockK, 0, 0, 2 * it.mb + (int)rank, it.e, full);
                         else
                             tma_load_3d_pair(sa, &map_a, ks * kBlockK, 256 * it.mb + 128 * (int)rank, it.e, full);
+                        if (DBL_ROWS > 0 && dbl) {  // the next block of weight rows behind it
+                            if (MODE == 1)
+                                tma_load_5d_pair(sa + kATileBytes, &map_a, ks * kBlockK, 0, 0, 2 * it.mb + 2 + (int)rank, it.e, full);
+                            else
+                                tma_load_3d_pair(sa + kATileBytes, &map_a, ks * kBlockK, 256 * it.mb + 256 + 128 * (int)rank, it.e, full);
+                        }
                     }
                     __syncwarp();
                 }
@@ -235,9 +267,8 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 s_abort = 1;
             }
         }
-    } else if (MODE == 2 && warp == 3) {
-        // ------------------------------------------------------------------ TMA producer of the Hmid rows (GEMM2)
-        // A second issuing warp: one cannot issue the loads of both operands fast enough.
+    } else if (b_prod >= 0) {
+        // ------------------------------------------------------------------ TMA producers of the Hmid rows (GEMM2)
         {
             uint32_t it_count = 0;
             bool ok = true;
@@ -247,12 +278,14 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 if (got <= 0) { ok = got == 0; break; }
                 const int half = ((it.n + 31) >> 5) << 4;
                 const int brow0 = (int)rank * half;  // first tile column / pair row this CTA loads
+                const uint32_t b_off = (double_item(DBL_ROWS, it.n, it.mb, m_blocks) ? 2 : 1) * kATileBytes;
                 for (int ks = 0; ks < k_steps; ++ks, ++it_count) {
+                    if ((int)(it_count % kProducers) != b_prod) continue;
                     const uint32_t s = it_count % STAGES, ph = (it_count / STAGES) & 1u;
                     ok = __all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag));
                     if (!ok) break;
                     const uint32_t full = full0 + 8 * s;
-                    const uint32_t sb = ring + s * kStageBytes + kATileBytes;
+                    const uint32_t sb = ring + s * kStageBytes + b_off;
                     if (elect_one()) {
                         int b = 0;
 #pragma unroll
@@ -286,26 +319,48 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 if (got <= 0) { ok = got == 0; break; }
                 const int n_cols = ((it.n + 31) >> 5) << 5;
                 const uint32_t idesc = instr_desc_pair(n_cols);
-                const uint32_t buf = ACC_BUFS == 2 ? (tile_count & 1u) : 0u;
-                const uint32_t tph = (ACC_BUFS == 2 ? (tile_count >> 1) : tile_count) & 1u;
+                const bool dbl = double_item(DBL_ROWS, it.n, it.mb, m_blocks);
+                const uint32_t buf = tile_count & 1u;
+                const uint32_t tph = (tile_count >> 1) & 1u;
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * buf, tph ^ 1u, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d = tmem_base + buf * kAccCols;
-                for (int ks = 0; ks < k_steps; ++ks) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph, abort_flag));
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint64_t a = a0 + (uint64_t)(s * (kStageBytes >> 4));
-                    const uint64_t b = b0 + (uint64_t)(s * (kStageBytes >> 4));
-                    if (elect_one()) {  // always the same lane: a commit covers the MMAs of the thread that issues it
+                if (DBL_ROWS > 0 && dbl) {
+                    for (int ks = 0; ks < k_steps; ++ks) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph, abort_flag));
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t a = a0 + (uint64_t)(s * (kStageBytes >> 4));
+                        const uint64_t b = b0 + (uint64_t)(s * (kStageBytes >> 4) + (kATileBytes >> 4));  // the pair rows follow the second weight tile
+                        if (elect_one()) {  // always the same lane: a commit covers the MMAs of the thread that issues it
 #pragma unroll
-                        for (int k = 0; k < kBlockK / 16; ++k)  // +32 bytes per 16-element k slice inside the swizzle row
-                            umma_bf16_pair(d, a + 2 * k, b + 2 * k, idesc, (ks | k) ? 1u : 0u);
-                        umma_commit_pair(bar_empty + 8 * s);  // the stage is free in both CTAs once these MMAs have read it
+                            for (int k = 0; k < kBlockK / 16; ++k) {  // +32 bytes per 16-element k slice inside the swizzle row
+                                umma_bf16_pair(d, a + 2 * k, b + 2 * k, idesc, (ks | k) ? 1u : 0u);
+                                // the second block of weight rows, into columns 128..
+                                umma_bf16_pair(d + 128, a + (kATileBytes >> 4) + 2 * k, b + 2 * k, idesc, (ks | k) ? 1u : 0u);
+                            }
+                            umma_commit_pair(bar_empty + 8 * s);  // the stage is free in both CTAs once these MMAs have read it
+                        }
+                        __syncwarp();
+                        if (++s == STAGES) { s = 0; ph ^= 1u; }
                     }
-                    __syncwarp();
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                } else {
+                    for (int ks = 0; ks < k_steps; ++ks) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, ph, abort_flag));
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t a = a0 + (uint64_t)(s * (kStageBytes >> 4));
+                        const uint64_t b = b0 + (uint64_t)(s * (kStageBytes >> 4));
+                        if (elect_one()) {  // always the same lane: a commit covers the MMAs of the thread that issues it
+#pragma unroll
+                            for (int k = 0; k < kBlockK / 16; ++k)  // +32 bytes per 16-element k slice inside the swizzle row
+                                umma_bf16_pair(d, a + 2 * k, b + 2 * k, idesc, (ks | k) ? 1u : 0u);
+                            umma_commit_pair(bar_empty + 8 * s);  // the stage is free in both CTAs once these MMAs have read it
+                        }
+                        __syncwarp();
+                        if (++s == STAGES) { s = 0; ph ^= 1u; }
+                    }
                 }
                 if (!ok) break;
                 if (elect_one()) umma_commit_pair(bar_tfull + 8 * buf);    // accumulators complete in both CTAs
@@ -367,10 +422,16 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 if (!ok) break;
                 bool end = false;
                 if (lane == 0) {
-                    const long long item = atomicAdd(counter, 1);
                     Item it = {0, 0, 1, 0};
-                    end = item >= n_items;
-                    if (!end) it = load_item(item, m_blocks, tile_rows, tile_expert, tile_row0, counts, offsets);
+                    for (;;) {
+                        const long long item = atomicAdd(counter, 1);
+                        end = item >= n_items;
+                        if (end) break;
+                        it = load_item(item, m_blocks, tile_rows, tile_expert, tile_row0, counts, offsets);
+                        // the odd block of a narrow tile belongs to the double item of the block before it
+                        if (!(DBL_ROWS > 0 && it.n <= DBL_ROWS && (it.mb & 1))) break;
+                    }
+                    if (end) it = Item{0, 0, 1, 0};
                     const unsigned long long rec = pack_item(seq, end, it);
                     asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(peer_queue + 8 * (seq % kItemSlots)), "l"(rec) : "memory");
                     *reinterpret_cast<volatile unsigned long long *>(&s_items[seq % kItemSlots]) = rec;
@@ -382,7 +443,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 s_abort = 1;
             }
         }
-    } else if (MODE == 1 && warp >= 8) {
+    } else if (MODE == 1 && warp >= 8 && warp < 12) {
         // ------------------------------------------------------------------ x-row gather (GEMM1)
         // Thread gt copies 16-byte chunk (gt & 7) of rows (gt >> 3) + 16 i, i = 0..7, of this CTA's
         // half of the tile's pair rows.  The chunk lands where the 128-byte swizzle puts it
@@ -399,6 +460,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             if (got <= 0) { ok = got == 0; break; }
             const int half = ((it.n + 31) >> 5) << 4;
             const int brow0 = (int)rank * half;
+            const uint32_t b_off = (double_item(DBL_ROWS, it.n, it.mb, m_blocks) ? 2 : 1) * kATileBytes;
             const __nv_bfloat16 *src[HALF_MAX / 16];
 #pragma unroll
             for (int i = 0; i < HALF_MAX / 16; ++i) {
@@ -412,7 +474,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                 if (lane == 0) ok = mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag);
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
-                const uint32_t sb = ring + s * kStageBytes + kATileBytes + dst_off;
+                const uint32_t sb = ring + s * kStageBytes + b_off + dst_off;
 #pragma unroll
                 for (int i = 0; i < HALF_MAX / 16; ++i)
                     if (rsub + 16 * i < half) cp_async16(sb + i * 16 * kRowBytes, src[i] + ks * kBlockK);
@@ -436,8 +498,8 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         for (uint32_t seq = 0; ok; ++seq, ++tile_count) {
             Item it;
             int status = next_item(queue, seq, it, abort_flag);  // 1 item, 0 end of the list, -1 gave up
-            const uint32_t buf = ACC_BUFS == 2 ? (tile_count & 1u) : 0u;
-            const uint32_t tph = (ACC_BUFS == 2 ? (tile_count >> 1) : tile_count) & 1u;
+            const uint32_t buf = tile_count & 1u;
+            const uint32_t tph = (tile_count >> 1) & 1u;
             if (status > 0 && !mbar_wait(bar_tfull + 8 * buf, tph, abort_flag)) status = -1;
             status = __reduce_min_sync(0xffffffffu, status);  // also reconverges the warp before the aligned TMEM loads
             if (MODE == 1) {
@@ -449,9 +511,12 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             }
             if (status <= 0) { ok = status == 0; break; }
             tc_fence_after();
-            const uint32_t t0 = tmem_base + ((uint32_t)(32 * q) << 16) + buf * kAccCols;
+            // one block of weight rows of the item: accumulator columns col0.., block mb; `last`: the
+            // buffer goes back to the MMA warp after this block's last read
+            auto drain = [&](uint32_t col0, int mb, bool last_sub) {
+            const uint32_t t0 = tmem_base + ((uint32_t)(32 * q) << 16) + buf * kAccCols + col0;
             if (MODE == 1) {
-                const int f0 = 128 * it.mb + 64 * (int)rank + 32 * wp;  // first of this warp's 32 features
+                const int f0 = 128 * mb + 64 * (int)rank + 32 * wp;  // first of this warp's 32 features
                 const bool f_ok = f0 < out_rows;
                 float *bw = xchg + (wp * 2 + (is_up ? 1 : 0)) * 1024;
                 const float *br = xchg + (wp * 2 + (is_up ? 0 : 1)) * 1024;
@@ -461,7 +526,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                     tmem_ld32_nowait(t0 + c0 + (is_up ? 0 : 32), send_u);
                     tmem_ld32_nowait(t0 + c0 + (is_up ? 32 : 0), keep_u);
                     tmem_ld_wait();
-                    if (c0 + 64 >= it.n) {
+                    if (last_sub && c0 + 64 >= it.n) {
                         // last read of this buffer: hand it back to the MMA warp before the stores
                         tc_fence_before();
                         __syncwarp();
@@ -488,12 +553,12 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                     named_sync(1 + wp, 64);  // the partner has read this step's values before the next step overwrites them
                 }
             } else {
-                const int row0 = 256 * it.mb + 128 * (int)rank + 32 * q;  // first of this warp's 32 output features
+                const int row0 = 256 * mb + 128 * (int)rank + 32 * q;  // first of this warp's 32 output features
                 const bool r_ok = row0 < out_rows;
                 for (int c0 = 0; c0 < it.n; c0 += 32) {
                     float v[32];
                     tmem_ld32(t0 + c0, v);
-                    if (c0 + 32 >= it.n) {
+                    if (last_sub && c0 + 32 >= it.n) {
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster(tempty0 + 8 * buf);
@@ -511,6 +576,13 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                     __syncwarp();
                 }
             }
+            };
+            if (DBL_ROWS > 0 && double_item(DBL_ROWS, it.n, it.mb, m_blocks)) {
+                drain(0, it.mb, false);
+                drain(128, it.mb + 1, true);
+            } else {
+                drain(0, it.mb, true);
+            }
         }
         if (!ok && lane == 0) {
             if (!*abort_flag) atomicExch(&meta[kMetaError], 13);
@@ -526,36 +598,37 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     }
 }
 
-template <int MODE, int HALF_MAX, int STAGES>
+template <int MODE, int HALF_MAX, int STAGES, int DBL_ROWS>
 constexpr int pair_smem_bytes() {
-    return STAGES * (kATileBytes + HALF_MAX * kRowBytes) + kPatchBytes + (MODE == 1 ? kXchgBytes : 0) + 1024;
+    return STAGES * StageBytes<HALF_MAX, DBL_ROWS>::value + kPatchBytes + (MODE == 1 ? kXchgBytes : 0) + 1024;
 }
 
 // One configuration of the kernel: its attribute set-up and its launch.
-template <int MODE, int HALF_MAX, int STAGES, int ACC_BUFS>
+template <int MODE, int HALF_MAX, int STAGES, int DBL_ROWS>
 struct PairKernel {
-    static constexpr int kSmem = pair_smem_bytes<MODE, HALF_MAX, STAGES>();
+    static constexpr int kSmem = pair_smem_bytes<MODE, HALF_MAX, STAGES, DBL_ROWS>();
     static bool prepare() {
-        return cudaFuncSetAttribute(expert_gemm_pair_kernel<MODE, HALF_MAX, STAGES, ACC_BUFS>,
+        return cudaFuncSetAttribute(expert_gemm_pair_kernel<MODE, HALF_MAX, STAGES, DBL_ROWS>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) == cudaSuccess;
     }
     template <typename... Args>
     static cudaError_t launch(const zeda_moe *h, cudaStream_t s, Args &&...args) {
-        const int ctas_per_sm = ACC_BUFS == 1 ? 2 : 1;
-        const int grid = (h->sm_count / 2) * 2 * ctas_per_sm;
-        return launch_kernel(h->pdl, expert_gemm_pair_kernel<MODE, HALF_MAX, STAGES, ACC_BUFS>, dim3(grid),
+        const int grid = (h->sm_count / 2) * 2;
+        return launch_kernel(h->pdl, expert_gemm_pair_kernel<MODE, HALF_MAX, STAGES, DBL_ROWS>, dim3(grid),
                              dim3(MODE == 1 ? kThreadsGather : kThreads), kSmem, s, std::forward<Args>(args)...);
     }
 };
 
 // small: at most 64 pair rows per expert (decode batches, T <= 64), a weight stream with many small
 // stages; big: tiles of up to 256 pair rows
-using Gemm1Small = PairKernel<1, 32, 9, 2>;
-using Gemm2Small = PairKernel<2, 32, 10, 2>;
-using Gemm1Mid = PairKernel<1, 64, 8, 2>;
-using Gemm2Mid = PairKernel<2, 64, 8, 2>;
-using Gemm1Big = PairKernel<1, 128, 6, 2>;
-using Gemm2Big = PairKernel<2, 128, 6, 2>;
+using Gemm1Small = PairKernel<1, 32, 9, 0>;
+using Gemm2Small = PairKernel<2, 32, 10, 0>;
+using Gemm1Mid = PairKernel<1, 64, 8, 0>;
+using Gemm2Mid = PairKernel<2, 64, 8, 0>;
+// GEMM1: five stages of 40 KB (a full tile's 16 + 16 KB, a double item's 16 + 16 + 8 KB) are what fits
+// beside the epilogue's staging; GEMM2 has room for six stages of 36 KB when double items stop at 64 rows.
+using Gemm1Big = PairKernel<1, 128, 5, 128>;
+using Gemm2Big = PairKernel<2, 128, 6, 64>;
 constexpr int kSmallRowsMax = 64;
 constexpr int kMidRowsPerExpert = 100;  // mean slots per candidate (T K / (N + N_Z)) up to which the mid geometry is used
 
