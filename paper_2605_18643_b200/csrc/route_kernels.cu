@@ -171,10 +171,14 @@ __device__ __forceinline__ void topk_gate_token(const float *__restrict__ row, i
     else if (gate_mode == ZEDA_GATE_RENORM_REAL) my_w = (my_idx < n_real && sum_real > 0.f) ? my_p / sum_real : 0.f;
 }
 
+// block_hist (optional): pass 1 of the counting sort done here.  Every slot on a normal expert adds 1
+// to its entry of the histogram of its block of kSortTokens tokens (integer adds: the counts do not
+// depend on their order).  The histograms must be zero on entry; the placement kernel that consumes
+// them zeroes them again.
 template <int RPL>
 __global__ void __launch_bounds__(256)
 topk_gate_kernel(const float *__restrict__ logits, int n_parts, int T, int n_real, int n_cand, int K, int gate_mode,
-                 int32_t *__restrict__ topk_idx, float *__restrict__ topk_w) {
+                 int32_t *__restrict__ topk_idx, float *__restrict__ topk_w, int32_t *__restrict__ block_hist) {
     pdl_launch_dependents();
     pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -187,11 +191,14 @@ topk_gate_kernel(const float *__restrict__ logits, int n_parts, int T, int n_rea
     if (lane < K) {
         topk_idx[(size_t)t * K + lane] = my_idx;
         topk_w[(size_t)t * K + lane] = my_w;
+        if (block_hist && (unsigned)my_idx < (unsigned)n_real)
+            atomicAdd(block_hist + (size_t)(t / kSortTokens) * n_real + my_idx, 1);
     }
 }
 
 // ---------------------------------------------------------------------------------------------
-// Counting sort, pass 1: per-CTA histogram of the normal-expert slots of kSortTokens tokens.
+// Counting sort, pass 1 as a kernel of its own (the paths that do not take it in the top-K kernel):
+// per-CTA histogram of the normal-expert slots of kSortTokens tokens.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 slot_hist_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real,
@@ -412,7 +419,7 @@ slot_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kPlaceWarps * 32)
 slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n_real, int nblk,
-                       const int32_t *__restrict__ block_hist, int32_t *__restrict__ counts,
+                       int32_t *__restrict__ block_hist, int32_t *__restrict__ counts,
                        int32_t *__restrict__ offsets, int32_t *__restrict__ n_pairs_out, int32_t *__restrict__ meta,
                        const WorkLists wl, int tile_rows, int32_t *__restrict__ perm, int32_t *__restrict__ perm_user,
                        int32_t *__restrict__ inv, int32_t *__restrict__ pair_token) {
@@ -461,6 +468,18 @@ slot_scan_place_kernel(const int32_t *__restrict__ topk_idx, int T, int K, int n
         }
     }
     __syncthreads();
+    // The histograms go back to zero for the next call's top-K kernel: the CTA that is last to have
+    // read them (a ticket, nobody waits) clears them and the ticket counter.
+    __shared__ int s_ticket;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_ticket = atomicAdd(meta + kMetaHistTicket, 1);
+    }
+    __syncthreads();
+    if (s_ticket == (int)gridDim.x - 1) {
+        for (int i = threadIdx.x; i < nblk * n_real; i += blockDim.x) block_hist[i] = 0;
+        if (threadIdx.x == 0) meta[kMetaHistTicket] = 0;
+    }
     finish_expert_scan(sh, n_real, T * K, counts, offsets, n_pairs_out, meta, wl, blockIdx.x == 0, blockIdx.x, gridDim.x, tile_rows);
     __syncthreads();
     int32_t *mine = pos + warp * n_real;
@@ -658,20 +677,24 @@ int launch_route_from_logits(const zeda_moe *h, const float *logits, int T, cons
 #undef ZEDA_CALL_SMALL
         launches = 1;
     } else {
+        // up to kFoldMaxBlocks sort blocks the top-K kernel counts the slots itself and one more launch
+        // scans and places; beyond, histogram, scan and placement are kernels of their own
+        const bool fold = nblk <= kFoldMaxBlocks;
+        int32_t *hist_in_topk = fold ? ws.block_hist : nullptr;
 #define ZEDA_CALL_TOPK(R) \
     launch_kernel(h->pdl, topk_gate_kernel<R>, dim3((T + 7) / 8), dim3(256), 0, s, logits, n_parts, T, c.n_real, n_cand, K, \
-                  c.gate_mode, ws.topk_idx, ws.topk_w)
+                  c.gate_mode, ws.topk_idx, ws.topk_w, hist_in_topk)
         ZEDA_RPL_DISPATCH(ZEDA_CALL_TOPK);
 #undef ZEDA_CALL_TOPK
-        launch_kernel(h->pdl, slot_hist_kernel, dim3(nblk), dim3(256), sizeof(int32_t) * c.n_real, s,
-                      (const int32_t *)ws.topk_idx, T, K, c.n_real, ws.block_hist);
-        if (nblk <= kFoldMaxBlocks) {
+        if (fold) {
             launch_kernel(h->pdl, slot_scan_place_kernel, dim3(nblk), dim3(kPlaceWarps * 32),
                           sizeof(int32_t) * ((kPlaceWarps + 1) * c.n_real + kScanSlabInts), s, (const int32_t *)ws.topk_idx, T, K, c.n_real,
-                          nblk, (const int32_t *)ws.block_hist, ws.counts, ws.offsets, out.n_pairs, ws.meta, wl, tile_rows, ws.perm,
+                          nblk, ws.block_hist, ws.counts, ws.offsets, out.n_pairs, ws.meta, wl, tile_rows, ws.perm,
                           out.perm, ws.inv, ws.pair_token);
-            launches = 3;
+            launches = 2;
         } else {
+            launch_kernel(h->pdl, slot_hist_kernel, dim3(nblk), dim3(256), sizeof(int32_t) * c.n_real, s,
+                          (const int32_t *)ws.topk_idx, T, K, c.n_real, ws.block_hist);
             expert_scan_kernel<<<1, 512, 0, s>>>(ws.block_hist, nblk, c.n_real, T * K, ws.counts, ws.offsets,
                                                  out.n_pairs, ws.meta, wl, tile_rows);
             slot_place_kernel<<<nblk, kPlaceWarps * 32, sizeof(int32_t) * kPlaceWarps * c.n_real, s>>>(

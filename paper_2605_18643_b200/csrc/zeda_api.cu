@@ -45,6 +45,10 @@ bool config_ok(const zeda_moe_config_t *c, const char **why) {
     return w == nullptr;
 }
 
+size_t hist_bytes(const zeda_moe_config_t &c) {
+    return (size_t)((c.max_tokens + kSortTokens - 1) / kSortTokens) * c.n_real * sizeof(int32_t);
+}
+
 // Walks the workspace layout; with base == nullptr it only measures.
 size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int *max_tiles) {
     size_t off = 0;
@@ -69,7 +73,7 @@ size_t carve(const zeda_moe_config_t &c, unsigned char *base, Workspace *ws, int
     w.inv = (int32_t *)take(slots * 4);
     w.perm = (int32_t *)take(slots * 4);
     w.pair_token = (int32_t *)take(slots * 4);
-    w.block_hist = (int32_t *)take(nblk * c.n_real * 4);
+    w.block_hist = (int32_t *)take(hist_bytes(c));
     w.counts = (int32_t *)take((size_t)c.n_real * 4);
     w.offsets = (int32_t *)take((size_t)(c.n_real + 1) * 4);
     w.meta = (int32_t *)take(kMetaCount * 4);
@@ -253,6 +257,10 @@ zeda_status_t zeda_moe_create(const zeda_moe_config_t *cfg, const float *router_
     }
     e = cudaMemset(h->ws.meta, 0, kMetaCount * 4);
     if (e != cudaSuccess) { delete h; return cuda_fail("cudaMemset(meta)", e); }
+    // the block histograms of the counting sort are zero between calls (the top-K kernel adds into them,
+    // the placement kernel clears them)
+    e = cudaMemset(h->ws.block_hist, 0, hist_bytes(*cfg));
+    if (e != cudaSuccess) { delete h; return cuda_fail("cudaMemset(block_hist)", e); }
     e = cudaDeviceSynchronize();
     if (e != cudaSuccess) { delete h; return cuda_fail("cudaDeviceSynchronize", e); }
     *out = h;
@@ -524,6 +532,10 @@ zeda_status_t zeda_moe_clear_error(zeda_moe_t *h, void *stream) {
     cudaError_t e = cudaSetDevice(h->cfg.device);
     if (e != cudaSuccess) return cuda_fail("cudaSetDevice", e);
     e = cudaMemsetAsync(h->ws.meta + kMetaError, 0, sizeof(int32_t), static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
+    // a call that failed between its top-K and placement kernels leaves counts in the block histograms
+    e = cudaMemsetAsync(h->ws.block_hist, 0, hist_bytes(h->cfg), static_cast<cudaStream_t>(stream));
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->ws.meta + kMetaHistTicket, 0, sizeof(int32_t), static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail("cudaMemsetAsync", e);
     return ZEDA_OK;
 }

@@ -26,6 +26,7 @@ enum MetaSlot {
     kMetaPairTiles = 7,  // entries of the expert kernels' tile list
     kMetaNextItem1 = 8,  // next unclaimed work item of the GEMM1 kernel (reset by the routing pass)
     kMetaNextItem2 = 9,  // the same for GEMM2
+    kMetaHistTicket = 10,  // placement CTAs that have read the block histograms (the last one clears them)
     kMetaCount = 16
 };
 
