@@ -171,7 +171,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     static_assert(DBL_ROWS <= 128 && DBL_ROWS % 32 == 0 && DBL_ROWS <= 2 * HALF_MAX, "two accumulators of a double item share 256 columns");
     constexpr int kStageBytes = StageBytes<HALF_MAX, DBL_ROWS>::value;
     constexpr int kTmemCols = 2 * kAccCols;
-    pdl_launch_dependents();
+    if (MODE == 2) pdl_launch_dependents();
     extern __shared__ __align__(1024) unsigned char pair_smem[];
     __shared__ __align__(8) unsigned long long bars[3 * STAGES + 4];
     __shared__ uint32_t s_tmem_base;
@@ -215,7 +215,15 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     tc_fence_after();
     const uint32_t tmem_base = s_tmem_base;
     volatile int *abort_flag = &s_abort;
-    pdl_wait();  // everything above is local set-up; the routing results and activations are read below
+    // Everything above is local set-up.  GEMM1 reads the routing results from here on, so it waits for
+    // its predecessor, and only then releases GEMM2: a GEMM2 CTA therefore never runs before the routing
+    // pass is complete, and of GEMM2's roles only the producers of the Hmid rows have to wait for
+    // GEMM1 itself.  The others (weight producers, scheduler) start on the first items as soon as the
+    // CTA is resident, under GEMM1's tail.
+    if (MODE == 1) {
+        pdl_wait();
+        pdl_launch_dependents();
+    }
 
     const int k_steps = kdim / kBlockK;
     const volatile unsigned long long *queue = s_items;
@@ -269,6 +277,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
         }
     } else if (b_prod >= 0) {
         // ------------------------------------------------------------------ TMA producers of the Hmid rows (GEMM2)
+        pdl_wait();  // Hmid is GEMM1's output
         {
             uint32_t it_count = 0;
             bool ok = true;
