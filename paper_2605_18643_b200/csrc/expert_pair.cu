@@ -10,11 +10,12 @@
 // most 128 activation rows per 128 x 256 block of outputs.
 //
 //   work item  = (expert e, block of <= 256 of its pair rows, block mb of weight rows)
-//   GEMM1      A tile of CTA r = 64 gate rows of 64-row block (2 mb + r) followed by the matching 64
-//              up rows (one 5-D TMA box); B = x rows of the pairs, fetched by four gather warps
-//              through pair_token with 16-byte cp.async into the 128-byte-swizzled layout; K = H.
-//              TMEM lanes 0-63 hold gate values, lanes 64-127 the up values of the same features;
-//              the epilogue warps swap halves through shared memory, apply SwiGLU and store Hmid.
+//   GEMM1      A tile of CTA r = the 64 features of 64-row block (2 mb + r) as four groups of 16 gate
+//              rows each followed by the matching 16 up rows (one 5-D TMA box); B = x rows of the
+//              pairs, fetched by four gather warps through pair_token with 16-byte cp.async into
+//              the 128-byte-swizzled layout; K = H.  An epilogue warp's 32 TMEM lanes thus hold the
+//              gate values (lanes 0-15) and the up values (lanes 16-31) of the same 16 features:
+//              the halves meet through one warp shuffle per column pair, SwiGLU, store of Hmid.
 //   GEMM2      A tile of CTA r = 128 down rows [256 mb + 128 r, +128); B = Hmid rows; K = H_e.
 //
 // One CTA per SM, persistent over a device-side work list (the host never learns P or the counts).
@@ -47,7 +48,6 @@ constexpr int kThreads = 320;                   // GEMM2: warps 8, 9 are the sec
 constexpr int kThreadsGather = 416;             // GEMM1: four gather warps, warp 12 the second weight issuer
 constexpr int kProducers = 2;                   // warps that share a TMA stream, k-step c going to warp c mod 2
 constexpr int kPatchBytes = 4 * 32 * 32 * 2;    // per epilogue warp: [32 pair rows][32 features] bf16, for 16-byte stores
-constexpr int kXchgBytes = 2 * 2 * 32 * 32 * 4; // GEMM1 gate/up swap: [warp pair][direction][32 cols][32 lanes] fp32
 
 // Hmid row blocks come in boxes of 128, 64, 32 and 16 rows: a block of 16 k rows is loaded with
 // at most four TMA instructions (few large boxes: issuing a TMA instruction costs a few hundred cycles).
@@ -56,7 +56,7 @@ struct RowMaps {
 };
 
 struct PairMaps {
-    CUtensorMap w_gate_up;  // [N][He/64 blocks][gate | up][64 rows][d]  box {64, 64, 2, 1, 1}
+    CUtensorMap w_gate_up;  // [N][He/16 groups][gate | up][16 rows][d]  box {64, 16, 2, 4, 1}
     CUtensorMap w_down;     // [N][d][He]   box {64, 128, 1}
     RowMaps hmid;           // [rows][He]
 };
@@ -138,10 +138,6 @@ __device__ __forceinline__ int next_item(const volatile unsigned long long *queu
     return 1;
 }
 
-__device__ __forceinline__ void named_sync(int id, int threads) {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
-
 __device__ __forceinline__ float swiglu(float g, float u) { return __fdividef(g * u, 1.f + __expf(-g)); }
 
 // A tile of at most DBL_ROWS pair rows takes two blocks of weight rows per item ("double item"): a
@@ -176,7 +172,6 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     __shared__ __align__(8) unsigned long long bars[3 * STAGES + 4];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
-    __shared__ int s_ok[4];
     __shared__ __align__(8) unsigned long long s_items[kItemSlots];  // this CTA's copy of the item queue
     __shared__ int s_prod_seq;                                       // item the weight producer is on (leader CTA)
 
@@ -184,7 +179,6 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     const uint32_t ring = (smem_u32(pair_smem) + 1023u) & ~1023u;
     unsigned char *after_ring = pair_smem + (ring - smem_u32(pair_smem)) + STAGES * kStageBytes;
     __nv_bfloat16 *patches = reinterpret_cast<__nv_bfloat16 *>(after_ring);
-    float *xchg = reinterpret_cast<float *>(after_ring + kPatchBytes);
     const uint32_t bar_full = smem_u32(&bars[0]);                 // used in the leader CTA only
     const uint32_t bar_empty = smem_u32(&bars[STAGES]);           // one set per CTA
     const uint32_t bar_tfull = smem_u32(&bars[2 * STAGES]);       // one set per CTA
@@ -256,13 +250,13 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
                     const uint32_t sa = ring + s * kStageBytes;
                     if (elect_one()) {
                         if (leader) mbar_expect_tx(bar_full + 8 * s, bytes);  // the TMA bytes of both CTAs
-                        if (MODE == 1)  // one box: 64 gate rows of block (2 mb + rank), then the 64 up rows of the same block
-                            tma_load_5d_pair(sa, &map_a, ks * kBlockK, 0, 0, 2 * it.mb + (int)rank, it.e, full);
+                        if (MODE == 1)  // one box: the 64 features of block (2 mb + rank), 16 gate rows then their 16 up rows, four times
+                            tma_load_5d_pair(sa, &map_a, ks * kBlockK, 0, 0, 4 * (2 * it.mb + (int)rank), it.e, full);
                         else
                             tma_load_3d_pair(sa, &map_a, ks * kBlockK, 256 * it.mb + 128 * (int)rank, it.e, full);
                         if (DBL_ROWS > 0 && dbl) {  // the next block of weight rows behind it
                             if (MODE == 1)
-                                tma_load_5d_pair(sa + kATileBytes, &map_a, ks * kBlockK, 0, 0, 2 * it.mb + 2 + (int)rank, it.e, full);
+                                tma_load_5d_pair(sa + kATileBytes, &map_a, ks * kBlockK, 0, 0, 4 * (2 * it.mb + 2 + (int)rank), it.e, full);
                             else
                                 tma_load_3d_pair(sa + kATileBytes, &map_a, ks * kBlockK, 256 * it.mb + 256 + 128 * (int)rank, it.e, full);
                         }
@@ -498,8 +492,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
     } else if (warp >= 4 && warp < 8) {
         // ------------------------------------------------------------------ epilogue warps
         const int q = warp & 3;      // TMEM lane quarter this warp may read
-        const int wp = q & 1;        // GEMM1: warp pair (gate warp q = wp, up warp q = wp + 2) sharing 32 features
-        const bool is_up = q >= 2;
+        const bool upper = lane >= 16;  // GEMM1: this lane holds up values; lane - 16 the gate values of the same feature
         __nv_bfloat16 *patch = patches + q * 1024;   // [32 pair rows][32 features]
         const int prow = lane >> 2, pch = lane & 3;  // 16-byte piece this lane stores: rows prow + 8 i, features 8 pch ..
         uint32_t tile_count = 0;
@@ -511,13 +504,6 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             const uint32_t tph = (tile_count >> 1) & 1u;
             if (status > 0 && !mbar_wait(bar_tfull + 8 * buf, tph, abort_flag)) status = -1;
             status = __reduce_min_sync(0xffffffffu, status);  // also reconverges the warp before the aligned TMEM loads
-            if (MODE == 1) {
-                // the two warps of a pair meet at named barriers below: they must leave the loop together
-                if (lane == 0) s_ok[q] = status;
-                named_sync(1 + wp, 64);
-                status = min(s_ok[wp], s_ok[wp + 2]);
-                named_sync(1 + wp, 64);
-            }
             if (status <= 0) { ok = status == 0; break; }
             tc_fence_after();
             // one block of weight rows of the item: accumulator columns col0.., block mb; `last`: the
@@ -525,41 +511,37 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
             auto drain = [&](uint32_t col0, int mb, bool last_sub) {
             const uint32_t t0 = tmem_base + ((uint32_t)(32 * q) << 16) + buf * kAccCols + col0;
             if (MODE == 1) {
-                const int f0 = 128 * mb + 64 * (int)rank + 32 * wp;  // first of this warp's 32 features
+                const int f0 = 128 * mb + 64 * (int)rank + 16 * q;  // first of this warp's 16 features
                 const bool f_ok = f0 < out_rows;
-                float *bw = xchg + (wp * 2 + (is_up ? 1 : 0)) * 1024;
-                const float *br = xchg + (wp * 2 + (is_up ? 0 : 1)) * 1024;
-                for (int c0 = 0; c0 < it.n; c0 += 64) {
-                    // the gate warp finishes columns [c0, c0+32), the up warp columns [c0+32, c0+64)
-                    uint32_t keep_u[32], send_u[32];
-                    tmem_ld32_nowait(t0 + c0 + (is_up ? 0 : 32), send_u);
-                    tmem_ld32_nowait(t0 + c0 + (is_up ? 32 : 0), keep_u);
+                for (int c0 = 0; c0 < it.n; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32_nowait(t0 + c0, v);
                     tmem_ld_wait();
-                    if (last_sub && c0 + 64 >= it.n) {
+                    if (last_sub && c0 + 32 >= it.n) {
                         // last read of this buffer: hand it back to the MMA warp before the stores
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster(tempty0 + 8 * buf);
                     }
+                    // Columns in pairs: the gate lane finishes the even column, the up lane the odd one;
+                    // one shuffle hands each the value it lacks.
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) bw[j * 32 + lane] = __uint_as_float(send_u[j]);
-                    named_sync(1 + wp, 64);
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const float other = br[j * 32 + lane];
-                        const float mine = __uint_as_float(keep_u[j]);
-                        patch[j * 32 + lane] = __float2bfloat16_rn(is_up ? swiglu(other, mine) : swiglu(mine, other));
+                    for (int i = 0; i < 16; ++i) {
+                        const float even = __uint_as_float(v[2 * i]), odd = __uint_as_float(v[2 * i + 1]);
+                        const float got = __shfl_xor_sync(0xffffffffu, upper ? even : odd, 16);
+                        const float h = upper ? swiglu(got, odd) : swiglu(even, got);
+                        patch[(2 * i + (upper ? 1 : 0)) * 16 + (lane & 15)] = __float2bfloat16_rn(h);  // [32 pair rows][16 features]
                     }
                     __syncwarp();
-                    const int cb = c0 + (is_up ? 32 : 0);
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int r = prow + 8 * i;
-                        const uint4 val = *reinterpret_cast<const uint4 *>(patch + r * 32 + pch * 8);
-                        if (f_ok && cb + r < it.n)
-                            *reinterpret_cast<uint4 *>(out + (size_t)(it.pos0 + cb + r) * out_ld + f0 + pch * 8) = val;
+                    for (int i = 0; i < 2; ++i) {
+                        const int piece = lane + 32 * i;  // 16-byte piece: pair row piece / 2, features 8 (piece & 1) ..
+                        const int r = piece >> 1;
+                        const uint4 val = *reinterpret_cast<const uint4 *>(patch + piece * 8);
+                        if (f_ok && c0 + r < it.n)
+                            *reinterpret_cast<uint4 *>(out + (size_t)(it.pos0 + c0 + r) * out_ld + f0 + (piece & 1) * 8) = val;
                     }
-                    named_sync(1 + wp, 64);  // the partner has read this step's values before the next step overwrites them
+                    __syncwarp();
                 }
             } else {
                 const int row0 = 256 * mb + 128 * (int)rank + 32 * q;  // first of this warp's 32 output features
@@ -609,7 +591,7 @@ expert_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
 
 template <int MODE, int HALF_MAX, int STAGES, int DBL_ROWS>
 constexpr int pair_smem_bytes() {
-    return STAGES * StageBytes<HALF_MAX, DBL_ROWS>::value + kPatchBytes + (MODE == 1 ? kXchgBytes : 0) + 1024;
+    return STAGES * StageBytes<HALF_MAX, DBL_ROWS>::value + kPatchBytes + 1024;
 }
 
 // One configuration of the kernel: its attribute set-up and its launch.
@@ -630,16 +612,19 @@ struct PairKernel {
 
 // small: at most 64 pair rows per expert (decode batches, T <= 64), a weight stream with many small
 // stages; big: tiles of up to 256 pair rows
-using Gemm1Small = PairKernel<1, 32, 9, 0>;
+using Gemm1Small = PairKernel<1, 32, 10, 0>;
 using Gemm2Small = PairKernel<2, 32, 10, 0>;
-using Gemm1Mid = PairKernel<1, 64, 8, 0>;
-using Gemm2Mid = PairKernel<2, 64, 8, 0>;
-// GEMM1: five stages of 40 KB (a full tile's 16 + 16 KB, a double item's 16 + 16 + 8 KB) are what fits
-// beside the epilogue's staging; GEMM2 has room for six stages of 36 KB when double items stop at 64 rows.
-using Gemm1Big = PairKernel<1, 128, 5, 128>;
+using Gemm1Mid = PairKernel<1, 64, 9, 0>;
+using Gemm2Mid = PairKernel<2, 64, 9, 0>;
+// Large tiles: six stages of 36 KB (a full tile's 16 + 16 KB, a double item of up to 64 pair rows
+// 16 + 16 + 4 KB).  GEMM1 has a second form for batches whose experts mostly hold 65..128 pairs: double
+// items up to 128 rows on five stages of 40 KB.
+using Gemm1Big = PairKernel<1, 128, 6, 64>;
+using Gemm1Wide = PairKernel<1, 128, 5, 128>;
 using Gemm2Big = PairKernel<2, 128, 6, 64>;
 constexpr int kSmallRowsMax = 64;
 constexpr int kMidRowsPerExpert = 100;  // mean slots per candidate (T K / (N + N_Z)) up to which the mid geometry is used
+constexpr int kWideRowsPerExpert = 256; // ... and up to which GEMM1 runs tiles of up to 128 rows as double items
 
 // The small geometry holds at most kSmallRowsMax pair rows of one expert.  Without expert parallelism
 // an expert has at most one pair per token of the call; with it, any number of the received rows.
@@ -669,11 +654,11 @@ int init_pair_kernels(zeda_moe *h) {
     const cuuint64_t rows = (cuuint64_t)h->pair_rows + kPairTileM;
     bool ok = true;
     {
-        // a 5-D view of [N][2 He][d] that lets one box fetch 64 gate rows and the matching 64 up rows:
-        // (k, row in block, gate | up, block of 64 rows, expert)
-        const cuuint64_t dims[5] = {d, 64, 2, He / 64, E};
-        const cuuint64_t strides[4] = {d * 2, He * d * 2, 64 * d * 2, 2 * He * d * 2};
-        const cuuint32_t box[5] = {kBlockK, 64, 2, 1, 1};
+        // a 5-D view of [N][2 He][d] that lets one box fetch 64 features as four groups of 16 gate rows
+        // each followed by the matching 16 up rows: (k, row in group, gate | up, group of 16 rows, expert)
+        const cuuint64_t dims[5] = {d, 16, 2, He / 16, E};
+        const cuuint64_t strides[4] = {d * 2, He * d * 2, 16 * d * 2, 2 * He * d * 2};
+        const cuuint32_t box[5] = {kBlockK, 16, 2, 4, 1};
         ok = ok && encode_bf16_map(&pm->w_gate_up, h->w_gate_up, 5, dims, strides, box);
     }
     {
@@ -689,7 +674,7 @@ int init_pair_kernels(zeda_moe *h) {
         ok = ok && encode_bf16_map(&pm->hmid.m[i], h->ws.hmid, 2, dims, strides, box);
     }
     ok = ok && Gemm1Small::prepare() && Gemm2Small::prepare() && Gemm1Mid::prepare() && Gemm2Mid::prepare() &&
-         Gemm1Big::prepare() && Gemm2Big::prepare();
+         Gemm1Big::prepare() && Gemm1Wide::prepare() && Gemm2Big::prepare();
     if (!ok) {
         free(pm);
         if (zeda_last_error()[0] == 0) set_error("pair kernel set-up failed: %s", cudaGetErrorString(cudaGetLastError()));
@@ -710,7 +695,9 @@ int launch_experts_gemm1_pair(const zeda_moe *h, const __nv_bfloat16 *x, const E
                                    w.tile_rows);
     };
     // an expert cannot hold more pair rows than the call has tokens (a token selects it at most once)
-    const cudaError_t e = small_geometry(h, w) ? go(Gemm1Small{}) : w.tile_rows == kMidTileM ? go(Gemm1Mid{}) : go(Gemm1Big{});
+    // (an expert-parallel rank does not know its load from the call's shape: it takes the form for large batches)
+    const bool wide = c.ep_size < 1 && (long long)w.rows_bound <= (long long)kWideRowsPerExpert * (c.n_real + c.n_zero);
+    const cudaError_t e = small_geometry(h, w) ? go(Gemm1Small{}) : w.tile_rows == kMidTileM ? go(Gemm1Mid{}) : wide ? go(Gemm1Wide{}) : go(Gemm1Big{});
     return e == cudaSuccess ? 1 : -1;
 }
 
