@@ -612,7 +612,7 @@ struct PairKernel {
 
 // small: at most 64 pair rows per expert (decode batches, T <= 64), a weight stream with many small
 // stages; big: tiles of up to 256 pair rows
-using Gemm1Small = PairKernel<1, 32, 10, 0>;
+using Gemm1Small = PairKernel<1, 32, 6, 64>;   // every tile of a small batch is a double item: 6 x (16 + 16 + 4 KB)
 using Gemm2Small = PairKernel<2, 32, 10, 0>;
 using Gemm1Mid = PairKernel<1, 64, 9, 0>;
 using Gemm2Mid = PairKernel<2, 64, 9, 0>;
